@@ -1,0 +1,161 @@
+/*
+ * fftconv -- FFT-domain convolution for CNN layers on NVIDIA B200 (sm_100a).
+ *
+ * C ABI of libfftconv.so.  Every pass is computed as the paper's Table 1
+ * pipeline: batched 2-D real-to-complex FFTs of the implicitly zero-padded
+ * planes, a per-frequency-bin complex contraction over the summed index, and
+ * an inverse complex-to-real FFT with crop and 1/n^2 scale.  All kernels are
+ * hand-written CUDA; there is no CPU fallback and no library call on the
+ * compute path.
+ *
+ * Notation (paper, Section 2): S minibatch, f input planes, fprime (f') output
+ * planes, h x w input plane, kh x kw kernel, oh x ow = (h-kh+1) x (w-kw+1)
+ * output plane ("valid" only), n = side of the square power-of-two Fourier
+ * basis, n >= max(h, w).
+ *
+ * Conventions for all entry points
+ *  - Data pointers are DEVICE pointers owned by the caller, fp32, contiguous
+ *    row-major ("BDHW", Section 3.1), at least 4-byte aligned (16-byte
+ *    alignment lets the loads vectorise):
+ *        x, dx [S][f][h][w]     w, dw [fprime][f][kh][kw]
+ *        y, dy [S][fprime][oh][ow]
+ *  - `cuda_stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *    Calls enqueue kernels on it and return; they never synchronise.  The conv
+ *    and transform calls allocate no device memory (the caller lends the plan
+ *    its workspace).
+ *  - Inputs are never modified.  The device used is the one current when the
+ *    call is made; plan, workspace and data must live on that device.
+ *  - Return value: FFTCONV_OK (0) or a negative fftconv_status.  Nothing is
+ *    thrown across the boundary.  On error no kernel has been launched.
+ */
+#ifndef FFTCONV_H_
+#define FFTCONV_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct conv_plan_s conv_plan_t; /* opaque; created and destroyed by the library */
+
+typedef enum {
+    FFTCONV_OK = 0,
+    FFTCONV_EINVAL = -1,        /* null pointer, non-positive count, kh > h, n < max(h, w) ... */
+    FFTCONV_EUNSUPPORTED = -2,  /* n not in {8,16,32,64,128}, unknown math mode            */
+    FFTCONV_EWORKSPACE = -3,    /* workspace missing, misaligned or too small              */
+    FFTCONV_ECUDA = -4,         /* a CUDA runtime / driver call failed                     */
+    FFTCONV_EDEVICE_TIMEOUT = -5 /* a bounded device-side wait ran out (status word set)   */
+} fftconv_status;
+
+typedef enum {
+    FFTCONV_MATH_AUTO = 0, /* tensor cores when the shape fills a tile, else FP32 */
+    FFTCONV_MATH_FP32 = 1, /* per-bin contraction with FP32 FFMA                  */
+    FFTCONV_MATH_TF32 = 2  /* per-bin contraction on tcgen05 tensor cores, TF32
+                              inputs, FP32 accumulation in tensor memory         */
+} fftconv_math;
+
+/* Plan for one layer shape (Section 3.4: one strategy per problem size, chosen
+ * once).  Host-only: validates the shape, picks kernels and sizes the
+ * workspace.  Needs no GPU.  *out receives the plan; destroy it with
+ * conv_plan_destroy.  EINVAL: null out, a count < 1, kh > h, kw > w,
+ * n < max(h, w).  EUNSUPPORTED: n not a power of two in [8, 128]. */
+int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, int w, int kh, int kw, int n);
+
+/* Select the arithmetic of the per-bin contraction (fftconv_math).  Changes the
+ * workspace size: query it again afterwards. */
+int conv_plan_set_math(conv_plan_t* plan, int math);
+
+/* Math mode the plan will actually run (FFTCONV_MATH_FP32 or _TF32) once AUTO is resolved. */
+int conv_plan_effective_math(const conv_plan_t* plan);
+
+/* Bytes of device scratch the three passes need: the frequency-domain copies of
+ * the two operands and of the result (Section 6 lists the same buffers), in the
+ * plan's private frequency-major layout.  0 on a null plan. */
+size_t conv_plan_workspace_bytes(const conv_plan_t* plan);
+
+/* Lend the plan `bytes` of device memory at `dev_ptr` (256-byte aligned).  The
+ * caller keeps ownership and must keep it alive while the plan is used.
+ * Contents need no initialisation and are overwritten by every pass.  Passes of
+ * one plan must not overlap in time (one workspace).  EWORKSPACE if too small
+ * or misaligned. */
+int conv_plan_set_workspace(conv_plan_t* plan, void* dev_ptr, size_t bytes);
+
+/* fprop (Section 2, first equation): y(s,j) = sum_i x(s,i) (star) w(j,i), valid
+ * cross-correlation.  Overwrites y [S][fprime][oh][ow]. */
+int conv_fprop(conv_plan_t* plan, const float* x, const float* w, float* y, void* cuda_stream);
+
+/* bprop (Section 2, second equation): dx(s,i) = sum_j dy(s,j) * w(j,i), full
+ * convolution.  Overwrites dx [S][f][h][w]. */
+int conv_bprop(conv_plan_t* plan, const float* dy, const float* w, float* dx, void* cuda_stream);
+
+/* accGrad (Section 2, third equation; index form in Section 6):
+ * dw(j,i) = sum_s dy(s,j) (star) x(s,i).  accumulate == 0 overwrites
+ * dw [fprime][f][kh][kw]; accumulate != 0 adds to it. */
+int conv_accgrad(conv_plan_t* plan, const float* dy, const float* x, float* dw, int accumulate,
+                 void* cuda_stream);
+
+/* Reads the plan's device status word (synchronises the device).  FFTCONV_OK,
+ * or FFTCONV_EDEVICE_TIMEOUT if a bounded wait inside a kernel gave up since
+ * the last call (the word is then cleared), or ECUDA. */
+int conv_plan_status(conv_plan_t* plan);
+
+/* Frees the plan (host memory and its timing events; never the workspace). */
+int conv_plan_destroy(conv_plan_t* plan);
+
+/* Per-stage device timing for benchmarks.  enable != 0 makes every following
+ * pass record CUDA events on its stream around each of its four kernels
+ * (forward FFT of the first operand, forward FFT of the second, per-bin
+ * contraction, inverse FFT -- the columns of the paper's Table 4 with the
+ * transposes fused away).  Creates the events on first use (the only state the
+ * plan owns on the device side). */
+int conv_plan_enable_stage_timing(conv_plan_t* plan, int enable);
+
+/* Waits for the last pass issued with timing enabled and writes the duration of
+ * its four kernels in milliseconds to out_ms[0..3].  EINVAL if timing is off or
+ * no pass has run. */
+int conv_plan_stage_times_ms(conv_plan_t* plan, float* out_ms);
+
+/* Bare batched 2-D real-to-complex transform (Supplement 8.2 definition,
+ * forward sign minus, unnormalised; Section 3.1 half-spectrum storage):
+ *   out[p][ky][kx] = sum_{r<h,c<w} in[p][r][c] exp(-2 pi i (ky r + kx c)/n)
+ * in : device [batch][h][w] fp32, zero-padded implicitly to n x n (never
+ *      materialised, Section 5.1).
+ * out: device [batch][n][n/2+1] interleaved (re, im) fp32 pairs, 8-byte aligned. */
+int fft2d_r2c(const float* in, void* out_c, int batch, int h, int w, int n, void* cuda_stream);
+
+/* Bare batched 2-D complex-to-real inverse transform with crop and scale
+ * (Section 3.1: the inverse transform's result is clipped):
+ *   out[p][r][c] (+)= scale * Re sum_{ky,kx<n} X~[p][ky][kx] exp(+2 pi i (ky r + kx c)/n)
+ * for r < oh, c < ow (window anchored at the origin), X~ the Hermitian
+ * extension of the stored half.  The input must be Hermitian-consistent (the
+ * spectrum of a real plane); otherwise the result is unspecified.
+ * in : device [batch][n][n/2+1] interleaved fp32 pairs.
+ * out: device [batch][oh][ow] fp32; accumulate != 0 adds to it. */
+int fft2d_c2r(const void* in_c, float* out, int batch, int n, int oh, int ow, float scale,
+              int accumulate, void* cuda_stream);
+
+/* Per-bin complex contraction alone (Table 1, the Cgemm row), exposed for
+ * testing and profiling: for every bin b,
+ *   C[b][m][nn] = sum_k A[b][m][k] * B[b][nn][k]         (no conjugation)
+ * Operands are planar: A is device [bins][2][M][lda] fp32 (plane 0 real, plane
+ * 1 imaginary, k contiguous, lda >= K), B likewise [bins][2][N][ldb], C
+ * [bins][2][M][ldc] with ldc >= N.  lda, ldb, ldc must be multiples of 4.
+ * math: FFTCONV_MATH_FP32 or FFTCONV_MATH_TF32 (AUTO resolves by shape).
+ * status_word: device int the kernel sets non-zero if a bounded wait gives up;
+ * may be NULL for the FP32 path. */
+int fftconv_bin_contract(const float* A, const float* B, float* C, int bins, int M, int N, int K,
+                         int lda, int ldb, int ldc, int math, int* status_word,
+                         void* cuda_stream);
+
+/* Text for a status code; never NULL. */
+const char* fftconv_status_string(int status);
+
+/* Number of kernel launches issued by this library since load (all plans, all
+ * threads); lets a benchmark state how many of this library's kernels ran. */
+unsigned long long fftconv_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FFTCONV_H_ */

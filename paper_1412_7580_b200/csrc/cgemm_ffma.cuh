@@ -1,0 +1,118 @@
+// Per-frequency-bin complex contraction with FP32 FFMA (Table 1, the Cgemm row).
+//
+// For every bin b:  C[b][m][n] = sum_k A[b][m][k] * B[b][n][k]   (complex, no
+// conjugation -- conjugates were folded into the forward FFT's store).
+// Operands are planar and k-contiguous: A is [bins][2][M][lda] (plane 0 real,
+// plane 1 imaginary), B is [bins][2][N][ldb], C is [bins][2][M][ldc].
+//
+// CTA tile 64 x 64 of one bin, 256 threads, each thread a 4 x 4 block of complex
+// outputs (64 FFMAs per k against four 16-byte shared loads).  This is the exact
+// fp32 path and the fallback for shapes too small for the tensor-core kernel.
+#pragma once
+
+#include <cuda_runtime.h>
+
+namespace fc {
+
+struct GemmParams {
+    const float* A;
+    const float* B;
+    float* C;
+    int bins, M, N, K;
+    int lda, ldb, ldc;
+};
+
+constexpr int FG_BM = 64, FG_BN = 64, FG_BK = 16, FG_PAD = 4, FG_T = 256;
+
+__global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
+    __shared__ __align__(16) float sA[2][FG_BK][FG_BM + FG_PAD];
+    __shared__ __align__(16) float sB[2][FG_BK][FG_BN + FG_PAD];
+
+    const int tid = threadIdx.x;
+    const int bin = blockIdx.z;
+    const int m_blk = blockIdx.y * FG_BM, n_blk = blockIdx.x * FG_BN;
+    const size_t planeA = (size_t)p.M * p.lda, planeB = (size_t)p.N * p.ldb,
+                 planeC = (size_t)p.M * p.ldc;
+    const float* Ab = p.A + (size_t)bin * 2 * planeA;
+    const float* Bb = p.B + (size_t)bin * 2 * planeB;
+    float* Cb = p.C + (size_t)bin * 2 * planeC;
+
+    const int tx = tid & 15, ty = tid >> 4;      // 16 x 16 threads
+    const int lk = tid & 15, lr = tid >> 4;      // loader: k within chunk, row group
+
+    float cr[4][4], ci[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) cr[i][j] = ci[i][j] = 0.0f;
+
+    for (int k0 = 0; k0 < p.K; k0 += FG_BK) {
+        // global -> shared, transposing to [k][row]; zero-fill outside M/N/K
+        const int k = k0 + lk;
+        const bool kin = k < p.K;
+#pragma unroll
+        for (int it = 0; it < FG_BM / 16; ++it) {
+            const int r = lr + 16 * it;
+            const int m = m_blk + r, n = n_blk + r;
+            float are = 0.f, aim = 0.f, bre = 0.f, bim = 0.f;
+            if (kin && m < p.M) {
+                are = __ldg(Ab + (size_t)m * p.lda + k);
+                aim = __ldg(Ab + planeA + (size_t)m * p.lda + k);
+            }
+            if (kin && n < p.N) {
+                bre = __ldg(Bb + (size_t)n * p.ldb + k);
+                bim = __ldg(Bb + planeB + (size_t)n * p.ldb + k);
+            }
+            sA[0][lk][r] = are; sA[1][lk][r] = aim;
+            sB[0][lk][r] = bre; sB[1][lk][r] = bim;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < FG_BK; ++kk) {
+            const float4 a_r = *reinterpret_cast<const float4*>(&sA[0][kk][ty * 4]);
+            const float4 a_i = *reinterpret_cast<const float4*>(&sA[1][kk][ty * 4]);
+            const float4 b_r = *reinterpret_cast<const float4*>(&sB[0][kk][tx * 4]);
+            const float4 b_i = *reinterpret_cast<const float4*>(&sB[1][kk][tx * 4]);
+            const float ar[4] = {a_r.x, a_r.y, a_r.z, a_r.w};
+            const float ai[4] = {a_i.x, a_i.y, a_i.z, a_i.w};
+            const float br[4] = {b_r.x, b_r.y, b_r.z, b_r.w};
+            const float bi[4] = {b_i.x, b_i.y, b_i.z, b_i.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    cr[i][j] = fmaf(ar[i], br[j], cr[i][j]);
+                    cr[i][j] = fmaf(-ai[i], bi[j], cr[i][j]);
+                    ci[i][j] = fmaf(ar[i], bi[j], ci[i][j]);
+                    ci[i][j] = fmaf(ai[i], br[j], ci[i][j]);
+                }
+        }
+        __syncthreads();
+    }
+
+    const int n0 = n_blk + tx * 4;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m_blk + ty * 4 + i;
+        if (m >= p.M) continue;
+        float* o_r = Cb + (size_t)m * p.ldc + n0;
+        float* o_i = o_r + planeC;
+        if (n0 + 3 < p.N) {
+            *reinterpret_cast<float4*>(o_r) = make_float4(cr[i][0], cr[i][1], cr[i][2], cr[i][3]);
+            *reinterpret_cast<float4*>(o_i) = make_float4(ci[i][0], ci[i][1], ci[i][2], ci[i][3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (n0 + j < p.N) { o_r[j] = cr[i][j]; o_i[j] = ci[i][j]; }
+        }
+    }
+}
+
+static cudaError_t launch_cgemm_ffma(const GemmParams& p, cudaStream_t st) {
+    dim3 grid((p.N + FG_BN - 1) / FG_BN, (p.M + FG_BM - 1) / FG_BM, p.bins);
+    if (grid.y > 65535u || grid.z > 65535u) return cudaErrorInvalidValue;
+    cgemm_ffma_kernel<<<grid, FG_T, 0, st>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace fc

@@ -1,0 +1,369 @@
+// C ABI of libfftconv.so: plans, the three convolution passes, the bare
+// transforms and the bare per-bin contraction.  Host code only validates,
+// sizes and launches; every step of the computation runs in the kernels of
+// fft_kernels.cuh, cgemm_ffma.cuh and cgemm_tc.cuh.
+#include "../../include/fftconv.h"
+
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+#include <cstring>
+#include <new>
+
+#include "cgemm_ffma.cuh"
+#include "cgemm_tc.cuh"
+#include "fft_kernels.cuh"
+
+#define FFTCONV_API extern "C" __attribute__((visibility("default")))
+
+namespace {
+
+std::atomic<unsigned long long> g_launches{0};
+
+constexpr size_t kAlign = 256;
+constexpr size_t kHeaderBytes = 256;   // workspace header: the device status word lives here
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int round4(int v) { return (v + 3) & ~3; }
+
+// One frequency-major matrix family: [bins][2][R][ld] floats.
+struct SpecDesc {
+    int R, C, ld;
+    size_t bytes(int bins) const { return (size_t)bins * 2 * R * ld * sizeof(float); }
+};
+
+// How one real tensor enters a pass: plane p of the BDHW tensor goes to matrix
+// position (row, col) with p = row*in_rs + col*in_cs.
+struct OperandDesc {
+    SpecDesc spec;
+    int h, w;               // plane size (forward) or crop window (inverse)
+    long long in_rs, in_cs;
+    int conj;
+};
+
+struct PassDesc {
+    OperandDesc a, b, c;    // c: result (h, w = crop window)
+    int M, N, K;            // per-bin contraction C[M][N] = sum_K A[M][K] B[N][K]
+};
+
+enum { PASS_FPROP = 0, PASS_BPROP = 1, PASS_ACCGRAD = 2 };
+
+}  // namespace
+
+struct conv_plan_s {
+    int S, f, fp, h, w, kh, kw, n;
+    int oh, ow, bins;
+    int math;          // requested fftconv_math
+    void* ws;
+    size_t ws_bytes;
+    int timing;             // record events around the four kernels of a pass
+    bool timed;             // a timed pass has been issued
+    cudaEvent_t ev[5];
+    bool ev_made;
+};
+
+namespace {
+
+// Operand roles per pass (Table 1 and Section 2; which operand carries the
+// conjugate follows from the convolution theorem for cross-correlation):
+//   fprop  : X^[b][s][i] , conj W^[b][j][i] -> Y^[b][s][j]     reduce over f
+//   bprop  : dY^[b][s][j],      W^[b][i][j] -> dX^[b][s][i]    reduce over f'
+//   accGrad: conj dY^[b][j][s], X^[b][i][s] -> dW^[b][j][i]    reduce over S
+PassDesc describe(const conv_plan_s& p, int pass) {
+    PassDesc d{};
+    auto spec = [](int R, int C) { return SpecDesc{R, C, round4(C)}; };
+    switch (pass) {
+        case PASS_FPROP:
+            d.a = {spec(p.S, p.f), p.h, p.w, p.f, 1, 0};
+            d.b = {spec(p.fp, p.f), p.kh, p.kw, p.f, 1, 1};
+            d.c = {spec(p.S, p.fp), p.oh, p.ow, 0, 0, 0};
+            d.M = p.S; d.N = p.fp; d.K = p.f;
+            break;
+        case PASS_BPROP:
+            d.a = {spec(p.S, p.fp), p.oh, p.ow, p.fp, 1, 0};
+            d.b = {spec(p.f, p.fp), p.kh, p.kw, 1, p.f, 0};      // w[j][i] -> row i, col j
+            d.c = {spec(p.S, p.f), p.h, p.w, 0, 0, 0};
+            d.M = p.S; d.N = p.f; d.K = p.fp;
+            break;
+        default:
+            d.a = {spec(p.fp, p.S), p.oh, p.ow, 1, p.fp, 1};     // dy[s][j] -> row j, col s
+            d.b = {spec(p.f, p.S), p.h, p.w, 1, p.f, 0};         // x[s][i]  -> row i, col s
+            d.c = {spec(p.fp, p.f), p.kh, p.kw, 0, 0, 0};
+            d.M = p.fp; d.N = p.f; d.K = p.S;
+            break;
+    }
+    return d;
+}
+
+int resolve_math(const conv_plan_s& p, const PassDesc& d) {
+    if (p.math == FFTCONV_MATH_FP32) return FFTCONV_MATH_FP32;
+    const bool fits = fc::tc_shape_supported(d.M, d.N, d.K);
+    if (p.math == FFTCONV_MATH_TF32) return fits ? FFTCONV_MATH_TF32 : FFTCONV_MATH_FP32;
+    return (fits && fc::tc_shape_profitable(d.M, d.N, d.K)) ? FFTCONV_MATH_TF32 : FFTCONV_MATH_FP32;
+}
+
+size_t pass_bytes(const conv_plan_s& p, int pass) {
+    PassDesc d = describe(p, pass);
+    return align_up(d.a.spec.bytes(p.bins), kAlign) + align_up(d.b.spec.bytes(p.bins), kAlign) +
+           align_up(d.c.spec.bytes(p.bins), kAlign);
+}
+
+bool valid_n(int n) { return n == 8 || n == 16 || n == 32 || n == 64 || n == 128; }
+
+int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, float* c_out,
+             int accumulate, cudaStream_t st) {
+    if (!plan || !a_in || !b_in || !c_out) return FFTCONV_EINVAL;
+    if (!plan->ws || plan->ws_bytes < conv_plan_workspace_bytes(plan)) return FFTCONV_EWORKSPACE;
+    const PassDesc d = describe(*plan, pass);
+    unsigned char* base = static_cast<unsigned char*>(plan->ws);
+    int* status = reinterpret_cast<int*>(base);
+    float* specA = reinterpret_cast<float*>(base + kHeaderBytes);
+    float* specB = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(specA) +
+                                            align_up(d.a.spec.bytes(plan->bins), kAlign));
+    float* specC = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(specB) +
+                                            align_up(d.b.spec.bytes(plan->bins), kAlign));
+
+    auto forward = [&](const OperandDesc& o, const float* in, float* spec) -> cudaError_t {
+        fc::FftParams fp{};
+        fp.real_in = in; fp.spec_out = spec;
+        fp.h = o.h; fp.w = o.w;
+        fp.R = o.spec.R; fp.C = o.spec.C; fp.ld = o.spec.ld;
+        fp.in_rs = o.in_rs; fp.in_cs = o.in_cs; fp.conj = o.conj;
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return fc::launch_r2c<fc::LAYOUT_FREQ_MAJOR>(plan->n, fp, st);
+    };
+    const bool timing = plan->timing && plan->ev_made;
+    auto mark = [&](int i) { if (timing) cudaEventRecord(plan->ev[i], st); };
+    mark(0);
+    if (forward(d.a, a_in, specA) != cudaSuccess) return FFTCONV_ECUDA;
+    mark(1);
+    if (forward(d.b, b_in, specB) != cudaSuccess) return FFTCONV_ECUDA;
+    mark(2);
+
+    fc::GemmParams gp{};
+    gp.A = specA; gp.B = specB; gp.C = specC;
+    gp.bins = plan->bins; gp.M = d.M; gp.N = d.N; gp.K = d.K;
+    gp.lda = d.a.spec.ld; gp.ldb = d.b.spec.ld; gp.ldc = d.c.spec.ld;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    cudaError_t ge;
+    if (resolve_math(*plan, d) == FFTCONV_MATH_TF32) ge = fc::launch_cgemm_tc(gp, status, st);
+    else ge = fc::launch_cgemm_ffma(gp, st);
+    if (ge != cudaSuccess) return FFTCONV_ECUDA;
+    mark(3);
+
+    fc::FftParams ip{};
+    ip.spec_in = specC; ip.real_out = c_out;
+    ip.h = d.c.h; ip.w = d.c.w;
+    ip.R = d.c.spec.R; ip.C = d.c.spec.C; ip.ld = d.c.spec.ld;
+    ip.scale = 1.0f / ((float)plan->n * (float)plan->n);
+    ip.accumulate = accumulate ? 1 : 0;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (fc::launch_c2r<fc::LAYOUT_FREQ_MAJOR>(plan->n, ip, st) != cudaSuccess) return FFTCONV_ECUDA;
+    mark(4);
+    if (timing) plan->timed = true;
+    return FFTCONV_OK;
+}
+
+}  // namespace
+
+FFTCONV_API int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, int w, int kh,
+                          int kw, int n) {
+    if (!out) return FFTCONV_EINVAL;
+    *out = nullptr;
+    if (S < 1 || f < 1 || fprime < 1 || h < 1 || w < 1 || kh < 1 || kw < 1 || n < 1)
+        return FFTCONV_EINVAL;
+    if (kh > h || kw > w) return FFTCONV_EINVAL;
+    if (!valid_n(n)) return FFTCONV_EUNSUPPORTED;
+    if (n < h || n < w) return FFTCONV_EINVAL;
+    // plane counts and per-tensor element counts must stay inside 31-bit grids / 63-bit offsets
+    const long long planes_max = 1LL << 30;
+    if ((long long)S * f > planes_max || (long long)S * fprime > planes_max ||
+        (long long)f * fprime > planes_max)
+        return FFTCONV_EUNSUPPORTED;
+    conv_plan_s* p = new (std::nothrow) conv_plan_s();
+    if (!p) return FFTCONV_EINVAL;
+    p->S = S; p->f = f; p->fp = fprime; p->h = h; p->w = w; p->kh = kh; p->kw = kw; p->n = n;
+    p->oh = h - kh + 1; p->ow = w - kw + 1;
+    p->bins = n * (n / 2 + 1);
+    p->math = FFTCONV_MATH_AUTO;
+    p->ws = nullptr; p->ws_bytes = 0;
+    p->timing = 0; p->timed = false; p->ev_made = false;
+    *out = p;
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_plan_set_math(conv_plan_t* plan, int math) {
+    if (!plan) return FFTCONV_EINVAL;
+    if (math != FFTCONV_MATH_AUTO && math != FFTCONV_MATH_FP32 && math != FFTCONV_MATH_TF32)
+        return FFTCONV_EUNSUPPORTED;
+    plan->math = math;
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_plan_effective_math(const conv_plan_t* plan) {
+    if (!plan) return FFTCONV_EINVAL;
+    // the mode all three passes share: TF32 only if every pass resolves to it
+    for (int pass = 0; pass < 3; ++pass)
+        if (resolve_math(*plan, describe(*plan, pass)) != FFTCONV_MATH_TF32) return FFTCONV_MATH_FP32;
+    return FFTCONV_MATH_TF32;
+}
+
+FFTCONV_API size_t conv_plan_workspace_bytes(const conv_plan_t* plan) {
+    if (!plan) return 0;
+    size_t m = 0;
+    for (int pass = 0; pass < 3; ++pass) {
+        size_t b = pass_bytes(*plan, pass);
+        if (b > m) m = b;
+    }
+    return kHeaderBytes + m;
+}
+
+FFTCONV_API int conv_plan_set_workspace(conv_plan_t* plan, void* dev_ptr, size_t bytes) {
+    if (!plan) return FFTCONV_EINVAL;
+    if (!dev_ptr || (reinterpret_cast<uintptr_t>(dev_ptr) % kAlign) != 0 ||
+        bytes < conv_plan_workspace_bytes(plan))
+        return FFTCONV_EWORKSPACE;
+    if (cudaMemset(dev_ptr, 0, kHeaderBytes) != cudaSuccess) return FFTCONV_ECUDA;
+    plan->ws = dev_ptr;
+    plan->ws_bytes = bytes;
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_fprop(conv_plan_t* plan, const float* x, const float* w, float* y,
+                           void* cuda_stream) {
+    return run_pass(plan, PASS_FPROP, x, w, y, 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
+FFTCONV_API int conv_bprop(conv_plan_t* plan, const float* dy, const float* w, float* dx,
+                           void* cuda_stream) {
+    return run_pass(plan, PASS_BPROP, dy, w, dx, 0, static_cast<cudaStream_t>(cuda_stream));
+}
+
+FFTCONV_API int conv_accgrad(conv_plan_t* plan, const float* dy, const float* x, float* dw,
+                             int accumulate, void* cuda_stream) {
+    return run_pass(plan, PASS_ACCGRAD, dy, x, dw, accumulate,
+                    static_cast<cudaStream_t>(cuda_stream));
+}
+
+FFTCONV_API int conv_plan_status(conv_plan_t* plan) {
+    if (!plan) return FFTCONV_EINVAL;
+    if (!plan->ws) return FFTCONV_EWORKSPACE;
+    if (cudaDeviceSynchronize() != cudaSuccess) return FFTCONV_ECUDA;
+    int word = 0;
+    if (cudaMemcpy(&word, plan->ws, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return FFTCONV_ECUDA;
+    if (word != 0) {
+        cudaMemset(plan->ws, 0, sizeof(int));
+        return FFTCONV_EDEVICE_TIMEOUT;
+    }
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_plan_destroy(conv_plan_t* plan) {
+    if (plan && plan->ev_made)
+        for (int i = 0; i < 5; ++i) cudaEventDestroy(plan->ev[i]);
+    delete plan;
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_plan_enable_stage_timing(conv_plan_t* plan, int enable) {
+    if (!plan) return FFTCONV_EINVAL;
+    if (enable && !plan->ev_made) {
+        for (int i = 0; i < 5; ++i)
+            if (cudaEventCreate(&plan->ev[i]) != cudaSuccess) {
+                for (int j = 0; j < i; ++j) cudaEventDestroy(plan->ev[j]);
+                return FFTCONV_ECUDA;
+            }
+        plan->ev_made = true;
+    }
+    plan->timing = enable ? 1 : 0;
+    plan->timed = false;
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_plan_stage_times_ms(conv_plan_t* plan, float* out_ms) {
+    if (!plan || !out_ms || !plan->timing || !plan->timed) return FFTCONV_EINVAL;
+    if (cudaEventSynchronize(plan->ev[4]) != cudaSuccess) return FFTCONV_ECUDA;
+    for (int i = 0; i < 4; ++i)
+        if (cudaEventElapsedTime(&out_ms[i], plan->ev[i], plan->ev[i + 1]) != cudaSuccess)
+            return FFTCONV_ECUDA;
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int fft2d_r2c(const float* in, void* out_c, int batch, int h, int w, int n,
+                          void* cuda_stream) {
+    if (!in || !out_c || batch < 1 || h < 1 || w < 1) return FFTCONV_EINVAL;
+    if (!valid_n(n)) return FFTCONV_EUNSUPPORTED;
+    if (n < h || n < w) return FFTCONV_EINVAL;
+    fc::FftParams p{};
+    p.real_in = in; p.spec_out = static_cast<float*>(out_c);
+    p.h = h; p.w = w; p.R = 1; p.C = batch; p.ld = batch;
+    p.in_rs = 0; p.in_cs = 1; p.conj = 0;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return fc::launch_r2c<fc::LAYOUT_BARE>(n, p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? FFTCONV_OK : FFTCONV_ECUDA;
+}
+
+FFTCONV_API int fft2d_c2r(const void* in_c, float* out, int batch, int n, int oh, int ow,
+                          float scale, int accumulate, void* cuda_stream) {
+    if (!in_c || !out || batch < 1 || oh < 1 || ow < 1) return FFTCONV_EINVAL;
+    if (!valid_n(n)) return FFTCONV_EUNSUPPORTED;
+    if (oh > n || ow > n) return FFTCONV_EINVAL;
+    fc::FftParams p{};
+    p.spec_in = static_cast<const float*>(in_c); p.real_out = out;
+    p.h = oh; p.w = ow; p.R = 1; p.C = batch; p.ld = batch;
+    p.scale = scale; p.accumulate = accumulate ? 1 : 0;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return fc::launch_c2r<fc::LAYOUT_BARE>(n, p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? FFTCONV_OK : FFTCONV_ECUDA;
+}
+
+FFTCONV_API int fftconv_bin_contract(const float* A, const float* B, float* C, int bins, int M,
+                                     int N, int K, int lda, int ldb, int ldc, int math,
+                                     int* status_word, void* cuda_stream) {
+    if (!A || !B || !C || bins < 1 || M < 1 || N < 1 || K < 1) return FFTCONV_EINVAL;
+    if (lda < K || ldb < K || ldc < N || (lda & 3) || (ldb & 3) || (ldc & 3)) return FFTCONV_EINVAL;
+    if (((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) |
+          reinterpret_cast<uintptr_t>(C)) & 15) != 0)
+        return FFTCONV_EINVAL;
+    if (bins > 65535) return FFTCONV_EUNSUPPORTED;
+    fc::GemmParams gp{};
+    gp.A = A; gp.B = B; gp.C = C;
+    gp.bins = bins; gp.M = M; gp.N = N; gp.K = K;
+    gp.lda = lda; gp.ldb = ldb; gp.ldc = ldc;
+    int eff = math;
+    if (math == FFTCONV_MATH_AUTO)
+        eff = (fc::tc_shape_supported(M, N, K) && fc::tc_shape_profitable(M, N, K))
+                  ? FFTCONV_MATH_TF32 : FFTCONV_MATH_FP32;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e;
+    if (eff == FFTCONV_MATH_TF32) {
+        if (!fc::tc_shape_supported(M, N, K)) return FFTCONV_EUNSUPPORTED;
+        if (!status_word) return FFTCONV_EINVAL;
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        e = fc::launch_cgemm_tc(gp, status_word, st);
+    } else if (eff == FFTCONV_MATH_FP32) {
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        e = fc::launch_cgemm_ffma(gp, st);
+    } else {
+        return FFTCONV_EUNSUPPORTED;
+    }
+    return e == cudaSuccess ? FFTCONV_OK : FFTCONV_ECUDA;
+}
+
+FFTCONV_API const char* fftconv_status_string(int status) {
+    switch (status) {
+        case FFTCONV_OK: return "ok";
+        case FFTCONV_EINVAL: return "invalid argument";
+        case FFTCONV_EUNSUPPORTED: return "unsupported size or mode";
+        case FFTCONV_EWORKSPACE: return "workspace missing, misaligned or too small";
+        case FFTCONV_ECUDA: return "CUDA call failed";
+        case FFTCONV_EDEVICE_TIMEOUT: return "bounded device-side wait ran out";
+    }
+    return "unknown status";
+}
+
+FFTCONV_API unsigned long long fftconv_launch_count(void) {
+    return g_launches.load(std::memory_order_relaxed);
+}

@@ -1,0 +1,147 @@
+"""The three convolution passes on the GPU against the float64 oracle.
+
+Tolerances (max |gpu - oracle| / max |oracle|): 1e-4 for the FP32 path, 5e-3
+for the TF32 tensor-core contraction.  Small shapes are compared element by
+element on full tensors; the benchmark-size layers are compared on a seeded
+sample of output coordinates (the oracle evaluates the plain definition at
+those coordinates) plus the adjoint identity on the full GPU tensors.
+"""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+TOL = {1: 1e-4, 2: 5e-3}   # MATH_FP32, MATH_TF32
+
+
+def relerr(got, ref):
+    m = np.max(np.abs(ref))
+    if m == 0:
+        return float(np.max(np.abs(got)))
+    return float(np.max(np.abs(got - ref)) / m)
+
+
+def run_gpu(shape, x, w, dy, math, accumulate_init=None):
+    import torch
+    import paper_1412_7580_b200 as fc
+    p = fc.conv_plan(*shape.args())
+    fc.conv_plan_set_math(p, math)
+    ws = fc.conv_plan_alloc_workspace(p)
+    ws.view(torch.float32)[64:].fill_(float("nan"))     # stale workspace must never leak
+    xd, wd, dyd = (torch.from_numpy(a).cuda() for a in (x, w, dy))
+    y = torch.full((shape.S, shape.fp, shape.oh, shape.ow), float("nan"), device="cuda")
+    dx = torch.full((shape.S, shape.f, shape.h, shape.w), float("nan"), device="cuda")
+    dw = torch.full((shape.fp, shape.f, shape.kh, shape.kw), float("nan"), device="cuda")
+    fc.conv_fprop(p, xd, wd, y)
+    fc.conv_bprop(p, dyd, wd, dx)
+    fc.conv_accgrad(p, dyd, xd, dw)
+    torch.cuda.synchronize()
+    assert fc.conv_plan_status(p) == 0
+    eff = fc.conv_plan_effective_math(p)
+    res = (y.cpu().numpy().astype(np.float64), dx.cpu().numpy().astype(np.float64),
+           dw.cpu().numpy().astype(np.float64), eff)
+    fc.conv_plan_destroy(p)
+    return res
+
+
+SMALL = [
+    # S, f, fp, h, w, kh, kw, n
+    (8, 4, 8, 16, 16, 3, 3, 16),       # the tiny benchmark config
+    (2, 3, 4, 8, 8, 3, 3, 8),
+    (1, 1, 1, 8, 8, 8, 8, 8),
+    (3, 5, 2, 7, 6, 3, 2, 8),
+    (5, 33, 17, 13, 13, 3, 3, 16),
+    (4, 7, 9, 16, 11, 5, 4, 16),
+    (3, 18, 20, 31, 31, 5, 5, 32),
+    (2, 5, 3, 27, 32, 7, 9, 32),
+    (9, 1, 16, 32, 32, 13, 13, 32),
+    (2, 9, 10, 64, 64, 11, 11, 64),
+    (3, 4, 1, 57, 57, 3, 3, 64),
+    (1, 2, 3, 128, 128, 13, 13, 128),
+    (2, 3, 2, 120, 120, 5, 5, 128),
+    (16, 16, 16, 13, 13, 3, 3, 16),
+    (1, 64, 1, 16, 16, 5, 5, 16),
+]
+
+
+@pytest.mark.parametrize("dims", SMALL)
+@pytest.mark.parametrize("math", [1, 2])
+def test_small_shapes_full_tensors(dims, math):
+    import oracle
+    from paper_1412_7580_b200 import workloads as wl
+    s = wl.ConvShape("case", *dims, cfg=7, point=sum(dims))
+    x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+    y, dx, dw, eff = run_gpu(s, x, w, dy, math)
+    tol = TOL[eff]
+    for got in (y, dx, dw):
+        assert np.all(np.isfinite(got))
+    assert relerr(y, oracle.fprop(x, w)) <= tol
+    assert relerr(dx, oracle.bprop(dy, w, s.h, s.w)) <= tol
+    assert relerr(dw, oracle.accgrad(dy, x, s.kh, s.kw)) <= tol
+
+
+def test_accgrad_accumulates():
+    import torch
+    import oracle
+    import paper_1412_7580_b200 as fc
+    from paper_1412_7580_b200 import workloads as wl
+    s = wl.ConvShape("acc", 4, 6, 5, 13, 13, 3, 3, 16, cfg=7, point=1)
+    x, dy = wl.make_x(s), wl.make_dy(s)
+    init = wl.make_w(s)
+    p = fc.conv_plan(*s.args())
+    fc.conv_plan_set_math(p, fc.MATH_FP32)
+    fc.conv_plan_alloc_workspace(p)
+    dw = torch.from_numpy(init.copy()).cuda()
+    fc.conv_accgrad(p, torch.from_numpy(dy).cuda(), torch.from_numpy(x).cuda(), dw, accumulate=True)
+    torch.cuda.synchronize()
+    ref = init.astype(np.float64) + oracle.accgrad(dy, x, s.kh, s.kw)
+    assert relerr(dw.cpu().numpy().astype(np.float64), ref) <= 1e-4
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3])
+@pytest.mark.parametrize("math", [1, 2])
+def test_benchmark_layers_sampled(cfg, math):
+    """Full-size layers in the launch configuration the benchmark times."""
+    import oracle
+    from paper_1412_7580_b200 import workloads as wl
+    s = wl.CONFIGS[cfg]
+    x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+    y, dx, dw, eff = run_gpu(s, x, w, dy, math)
+    tol = TOL[eff]
+    for got in (y, dx, dw):
+        assert np.all(np.isfinite(got))
+    # normalisation: max-abs of the sampled oracle values (close to the tensor's)
+    cy = wl.sample_coords(y.shape, 4000, seed=cfg)
+    ry = oracle.fprop_at(x, w, cy)
+    assert relerr(y[cy[:, 0], cy[:, 1], cy[:, 2], cy[:, 3]], ry) <= tol
+    cx = wl.sample_coords(dx.shape, 4000, seed=cfg + 10)
+    rx = oracle.bprop_at(dy, w, s.h, s.w, cx)
+    assert relerr(dx[cx[:, 0], cx[:, 1], cx[:, 2], cx[:, 3]], rx) <= tol
+    cw = wl.sample_coords(dw.shape, 600, seed=cfg + 20)
+    rw = oracle.accgrad_at(dy, x, s.kh, s.kw, cw)
+    assert relerr(dw[cw[:, 0], cw[:, 1], cw[:, 2], cw[:, 3]], rw) <= tol
+    # adjoint identity on the full GPU tensors: <y,dy> = <x,dx> = <w,dw>
+    a = float(np.sum(y * dy)); b = float(np.sum(dx * x)); c = float(np.sum(dw * w))
+    scale = np.sqrt(float(np.sum(y * y)) * float(np.sum(dy.astype(np.float64) ** 2)))
+    assert abs(a - b) <= 10 * tol * scale and abs(a - c) <= 10 * tol * scale
+
+
+def test_sweep_subset():
+    """A seeded slice of the parameter sweep (small enough for the CPU oracle
+    on sampled coordinates), all three passes, default math mode."""
+    import oracle
+    from paper_1412_7580_b200 import workloads as wl
+    pts = [s for s in wl.sweep_points(1000) if s.S * s.f * s.fp <= 16 * 64 * 64][:40]
+    assert len(pts) >= 20
+    for s in pts:
+        x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+        y, dx, dw, eff = run_gpu(s, x, w, dy, 0)
+        tol = TOL[eff]
+        cy = wl.sample_coords(y.shape, 300, seed=s.point)
+        assert relerr(y[cy[:, 0], cy[:, 1], cy[:, 2], cy[:, 3]], oracle.fprop_at(x, w, cy)) <= tol, s
+        cx = wl.sample_coords(dx.shape, 300, seed=s.point + 1)
+        assert relerr(dx[cx[:, 0], cx[:, 1], cx[:, 2], cx[:, 3]],
+                      oracle.bprop_at(dy, w, s.h, s.w, cx)) <= tol, s
+        cw = wl.sample_coords(dw.shape, 60, seed=s.point + 2)
+        assert relerr(dw[cw[:, 0], cw[:, 1], cw[:, 2], cw[:, 3]],
+                      oracle.accgrad_at(dy, x, s.kh, s.kw, cw)) <= tol, s
