@@ -1,0 +1,390 @@
+#!/usr/bin/env python
+"""Benchmark of the FFT-convolution hot path: one step = fprop + bprop + accGrad
+of one layer (all four kernels of each pass) on seeded synthetic tensors.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1] [--math auto]
+    python bench.py --impl reference ...     # the float64 CPU oracle on the host cores
+
+Prints ONE JSON line.  `value` is the paper's throughput metric (equivalent
+time-domain multiply-adds per second, Section 4.2, times two flops) summed over
+the three passes, with the inputs resident in HBM; `e2e` is the same metric with
+the host<->device copies inside the timed region; `roofline` describes the
+kernel with the largest share of the step; `cpu_baseline` is the oracle timed
+on a bounded sample of the same workload.  Under torchrun every rank runs the
+same layer on its own minibatch (data parallel over S: fprop and bprop need no
+exchange, the weight gradient is summed with one NCCL all-reduce).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "conv_gflops_equivalent_3pass"
+UNIT = "GFLOP/s-equivalent"
+FP32_FFMA_TFLOPS_NOMINAL = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x lanes x 2 flops x max clock
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------
+# Algorithmic bytes / flops of one pass (each real tensor and each spectrum
+# crosses HBM once in the FFT stages; the contraction reads two spectra and
+# writes one).
+# ---------------------------------------------------------------------------
+def pass_model(s, which):
+    B = s.n * (s.n // 2 + 1)
+    x_el, w_el, y_el = s.S * s.f * s.h * s.w, s.fp * s.f * s.kh * s.kw, s.S * s.fp * s.oh * s.ow
+    x_pl, w_pl, y_pl = s.S * s.f, s.fp * s.f, s.S * s.fp
+    if which == "fprop":
+        a, b, c = (x_el, x_pl), (w_el, w_pl), (y_el, y_pl)
+    elif which == "bprop":
+        a, b, c = (y_el, y_pl), (w_el, w_pl), (x_el, x_pl)
+    else:
+        a, b, c = (y_el, y_pl), (x_el, x_pl), (w_el, w_pl)
+    spec = lambda planes: planes * B * 8
+    stage_bytes = [a[0] * 4 + spec(a[1]), b[0] * 4 + spec(b[1]),
+                   spec(a[1]) + spec(b[1]) + spec(c[1]), spec(c[1]) + c[0] * 4]
+    return {
+        "stage_bytes": stage_bytes,                         # fft A, fft B, contraction, ifft
+        "b_fft": stage_bytes[0] + stage_bytes[1] + stage_bytes[3],
+        "b_gemm": stage_bytes[2],
+        "gemm_flops": 8.0 * s.S * s.f * s.fp * B,
+        "equiv_flops": 2.0 * s.macs,
+    }
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.uuid, self.proc, self.lines = uuid, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", self.uuid, "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.12] or [l for (_, l) in self.lines]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            parts = [p.strip() for p in l.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------
+# CPU oracle legs
+# ---------------------------------------------------------------------------
+def oracle_sample_run(s, x, w, dy, budget_s):
+    """Times the oracle (as it stands) on a bounded sample of output elements of
+    each pass; returns (equivalent flops done, seconds, description)."""
+    import oracle
+    from paper_1412_7580_b200 import workloads as wl
+    per = {"fprop": s.f * s.kh * s.kw, "bprop": s.fp * s.kh * s.kw, "accgrad": s.S * s.oh * s.ow}
+    dims = {"fprop": (s.S, s.fp, s.oh, s.ow), "bprop": (s.S, s.f, s.h, s.w),
+            "accgrad": (s.fp, s.f, s.kh, s.kw)}
+    fns = {"fprop": lambda c: oracle.fprop_at(x, w, c),
+           "bprop": lambda c: oracle.bprop_at(dy, w, s.h, s.w, c),
+           "accgrad": lambda c: oracle.accgrad_at(dy, x, s.kh, s.kw, c)}
+    total_macs, total_t, desc = 0.0, 0.0, []
+    for name in ("fprop", "bprop", "accgrad"):
+        # calibrate on a small sample, then size the timed sample to the budget
+        c0 = wl.sample_coords(dims[name], 2048, seed=1)
+        t = time.perf_counter(); fns[name](c0); dt = max(time.perf_counter() - t, 1e-6)
+        rate = len(c0) / dt
+        nel = int(min(max(rate * budget_s / 3.0, 2048), 50_000_000))
+        c = wl.sample_coords(dims[name], nel, seed=2)
+        t = time.perf_counter(); fns[name](c); dt = time.perf_counter() - t
+        # bprop border elements have fewer valid taps; count the formula's nominal taps
+        total_macs += float(len(c)) * per[name]
+        total_t += dt
+        desc.append("%s:%d elems" % (name, len(c)))
+    return 2.0 * total_macs, total_t, ", ".join(desc)
+
+
+def run_reference(args, s):
+    """--impl reference: the float64 oracle on the host cores, bounded sample per step."""
+    import oracle
+    from paper_1412_7580_b200 import workloads as wl
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+    cores = oracle.num_threads()
+    per_step = 3.0
+    for _ in range(args.warmup):
+        oracle_sample_run(s, x, w, dy, 0.3)
+    vals, times, desc = [], [], ""
+    for _ in range(args.steps):
+        fl, t, desc = oracle_sample_run(s, x, w, dy, per_step)
+        vals.append(fl / t / 1e9); times.append(t)
+    vals.sort()
+    v = vals[len(vals) // 2]
+    line = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * sum(times) / max(len(times), 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": s.name, "sample": "per step: " + desc},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "per step: " + desc},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------
+def run_ours(args, s):
+    import numpy as np
+    import torch
+    import paper_1412_7580_b200 as fc
+    from paper_1412_7580_b200 import workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    peaks = load_peaks()
+    math = {"auto": fc.MATH_AUTO, "fp32": fc.MATH_FP32, "tf32": fc.MATH_TF32}[args.math]
+    x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+    plan = fc.conv_plan(*s.args())
+    fc.conv_plan_set_math(plan, math)
+    ws = fc.conv_plan_alloc_workspace(plan)
+    eff = fc.conv_plan_effective_math(plan)
+    hx, hw_, hdy = (torch.from_numpy(a).pin_memory() for a in (x, w, dy))
+    xd, wd, dyd = hx.cuda(), hw_.cuda(), hdy.cuda()
+    y = torch.empty((s.S, s.fp, s.oh, s.ow), device="cuda")
+    dx = torch.empty((s.S, s.f, s.h, s.w), device="cuda")
+    dw = torch.empty((s.fp, s.f, s.kh, s.kw), device="cuda")
+    hy, hdx, hdw = (torch.empty(t.shape, dtype=torch.float32).pin_memory() for t in (y, dx, dw))
+
+    def step():
+        fc.conv_fprop(plan, xd, wd, y)
+        fc.conv_bprop(plan, dyd, wd, dx)
+        fc.conv_accgrad(plan, dyd, xd, dw)
+        if dist is not None:
+            dist.all_reduce(dw)        # data parallel over S: sum of the per-rank weight gradients
+
+    def step_e2e():
+        xd.copy_(hx, non_blocking=True); wd.copy_(hw_, non_blocking=True)
+        dyd.copy_(hdy, non_blocking=True)
+        step()
+        hy.copy_(y, non_blocking=True); hdx.copy_(dx, non_blocking=True)
+        hdw.copy_(dw, non_blocking=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", ""))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    launches0 = fc.fftconv_launch_count()
+    t0 = time.time()
+    ms_total = timed(step, args.steps)
+    # keep the GPU under the same load a little longer so the clock sampler sees it
+    reps = 0
+    while time.time() - t0 < 1.0 and reps < 200:
+        step(); reps += 1
+    torch.cuda.synchronize()
+    t1 = time.time()
+    launches = 12 * args.steps
+    assert fc.fftconv_launch_count() - launches0 == 12 * (args.steps + reps)
+    clocks = sampler.stop(t0, t1) if rank == 0 else None
+    ms_step = ms_total / args.steps
+
+    for _ in range(2):
+        step_e2e()
+    ms_e2e = timed(step_e2e, args.steps) / args.steps
+    assert fc.conv_plan_status(plan) == 0
+
+    flops_step = 3 * 2.0 * s.macs
+    value = world * flops_step / (ms_step * 1e-3) / 1e9
+    e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e9
+
+    # per-kernel durations from CUDA events recorded by the library on its stream
+    fc.conv_plan_enable_stage_timing(plan, True)
+    names = ["fprop", "bprop", "accgrad"]
+    calls = [lambda: fc.conv_fprop(plan, xd, wd, y), lambda: fc.conv_bprop(plan, dyd, wd, dx),
+             lambda: fc.conv_accgrad(plan, dyd, xd, dw)]
+    stage_ms = {n: np.zeros(4) for n in names}
+    pass_ms = {n: [] for n in names}
+    reps = max(args.steps, 10)
+    for _ in range(reps):
+        for n, c in zip(names, calls):
+            c()
+            t = np.array(fc.conv_plan_stage_times_ms(plan))
+            stage_ms[n] += t
+            pass_ms[n].append(float(t.sum()))
+    fc.conv_plan_enable_stage_timing(plan, False)
+    for n in names:
+        stage_ms[n] /= reps
+
+    tf32_peak = peaks["bf16_tflops_sustained"] / 2.0
+    p_tflops = tf32_peak if eff == fc.MATH_TF32 else FP32_FFMA_TFLOPS_NOMINAL
+    bw = peaks["hbm_gbs"] * 1e9
+    passes, best = {}, None
+    stage_names = ["r2c_fft_A", "r2c_fft_B", "bin_contraction", "c2r_ifft"]
+    for n in names:
+        m = pass_model(s, n)
+        t_ms = float(np.median(pass_ms[n]))
+        t_roof = max(m["b_fft"] / bw, m["gemm_flops"] / (p_tflops * 1e12))
+        t_stage = max((m["b_fft"] + m["b_gemm"]) / bw, m["gemm_flops"] / (p_tflops * 1e12))
+        passes[n] = {
+            "ms": t_ms, "gflops_equiv": m["equiv_flops"] / (t_ms * 1e-3) / 1e9,
+            "roofline_us": t_roof * 1e6, "roofline_frac": t_roof / (t_ms * 1e-3),
+            "unfused_roofline_us": t_stage * 1e6, "unfused_roofline_frac": t_stage / (t_ms * 1e-3),
+            "stage_ms": {k: float(v) for k, v in zip(stage_names, stage_ms[n])},
+        }
+        for k in range(4):
+            cand = (float(stage_ms[n][k]), n, k, m)
+            if best is None or cand[0] > best[0]:
+                best = cand
+    dur_ms, bn, bk, bm = best
+    if bk == 2 and bm["gemm_flops"] / (p_tflops * 1e12) > bm["stage_bytes"][2] / bw:
+        ach = bm["gemm_flops"] / (dur_ms * 1e-3) / 1e12
+        roof = {"bound": "tensor" if eff == fc.MATH_TF32 else "alu", "achieved": ach,
+                "peak": p_tflops, "unit": "TFLOP/s", "frac": ach / p_tflops}
+    else:
+        ach = bm["stage_bytes"][bk] / (dur_ms * 1e-3) / 1e9
+        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": ach / peaks["hbm_gbs"]}
+    roof.update({"traffic": None, "kernel": "%s/%s" % (bn, stage_names[bk]),
+                 "kernel_ms": dur_ms, "algorithmic_bytes": bm["stage_bytes"][bk],
+                 "peak_source": peaks["source"] + (" sustained bf16 / 2" if roof["bound"] == "tensor" else "")})
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        fl, t, desc = oracle_sample_run(s, x, w, dy, args.cpu_budget)
+        cpu = {"value": fl / t / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": desc + " (sampled output elements of each pass, plain definition, float64)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "tf32" if eff == fc.MATH_TF32 else "f32", "data": "synthetic",
+            "config": {"workload": s.name, "S": s.S, "f": s.f, "fprime": s.fp, "h": s.h, "w": s.w,
+                       "kh": s.kh, "kw": s.kw, "n": s.n, "passes": "fprop+bprop+accgrad",
+                       "parallelism": "dp%d over S" % world,
+                       "l2": "working set %.0f MB > 126 MB L2, no flush" % (
+                           (ws.numel() + 4 * (x.size + w.size + dy.size) * 2) / 1e6)},
+            "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e,
+                    "h2d_bytes_per_step": int(4 * (x.size + w.size + dy.size)),
+                    "d2h_bytes_per_step": int(4 * (y.numel() + dx.numel() + dw.numel()))},
+            "gpu_launches": launches, "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
+            "passes": passes,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=1, help="0 tiny, 1 mid (default), 2 large-kernel, 3 deep")
+    ap.add_argument("--math", default="auto", choices=["auto", "fp32", "tf32"])
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_1412_7580_b200 import workloads as wl
+    s = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, s)
+    else:
+        run_ours(args, s)
+
+
+if __name__ == "__main__":
+    main()
