@@ -1,9 +1,384 @@
-// placeholder until the tensor-core contraction lands
+// Per-frequency-bin complex contraction on the 5th-generation tensor cores
+// (Table 1, the Cgemm row): for every bin b,
+//     C[b][m][n] = sum_k A[b][m][k] * B[b][n][k]          (complex)
+// with planar, k-contiguous operands (see cgemm_ffma.cuh for the layout).
+//
+// The complex product is four real TF32 MMAs per k-step into two FP32
+// accumulators in tensor memory,
+//     C_re += A_re B_re ; C_re += (-A_im) B_im ; C_im += A_re B_im ; C_im += A_im B_re,
+// the minus sign coming from the instruction descriptor's negate-A bit, so no
+// expanded or interleaved copy of an operand is ever built.
+//
+// One persistent CTA per SM, warp-specialised:
+//   warp 0      TMA producer: 128-byte-swizzled boxes of 32 k-values x 128 rows
+//               of A_re, A_im, B_re, B_im per stage (64 KB), 3 stages in flight;
+//   warp 1      issues tcgen05.mma (one lane), owns the TMEM allocation;
+//   warps 2..5  epilogue: tcgen05.ld of the finished accumulators and stores to
+//               the frequency-major result, overlapped with the next tile's MMAs
+//               through two accumulator buffers (2 x 256 TMEM columns).
+// The per-bin problems are small and the kernel streams: it is bound by HBM
+// bytes (two spectra in, one out), not by tensor throughput.
+//
+// Every wait on an mbarrier is bounded; when one runs out the kernel raises the
+// caller's status word, drains what it issued, frees its tensor memory and
+// returns normally.
 #pragma once
+
+#include <cuda.h>
 #include <cuda_runtime.h>
+#include <stdint.h>
+
 #include "cgemm_ffma.cuh"
+
 namespace fc {
-static inline bool tc_shape_supported(int, int, int) { return false; }
-static inline bool tc_shape_profitable(int, int, int) { return false; }
-static cudaError_t launch_cgemm_tc(const GemmParams&, int*, cudaStream_t) { return cudaErrorNotSupported; }
+
+constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 32, TC_STAGES = 3;
+constexpr int TC_THREADS = 192;
+constexpr uint32_t TC_TILE_BYTES = TC_BM * TC_BK * 4;            // one 128 x 32 fp32 box: 16 KB
+constexpr uint32_t TC_STAGE_BYTES = 4 * TC_TILE_BYTES;           // A_re, A_im, B_re, B_im
+constexpr uint32_t TC_SMEM_BYTES = 1024 + TC_STAGES * TC_STAGE_BYTES + 256;
+constexpr uint32_t TC_TMEM_COLS = 512;
+constexpr long long TC_WAIT_CYCLES = 2000000000LL;               // about one second
+
+struct TcParams {
+    float* C;
+    int bins, M, N, K, ldc;
+    int m_tiles, n_tiles, k_blocks;
+    int* status;
+};
+
+static inline bool tc_shape_supported(int M, int N, int K) {
+    return M >= 1 && N >= 1 && K >= 1;
 }
+// Below these sizes most of a 128 x 128 x 32 tile would be padding.
+static inline bool tc_shape_profitable(int M, int N, int K) {
+    return M >= 32 && N >= 32 && K >= 16;
+}
+
+// ---- PTX wrappers ----------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > TC_WAIT_CYCLES) return false;
+    }
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                            int c2, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before_sync() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after_sync() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                            uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32"
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15,"
+        " %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31},"
+        " [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]),
+          "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]),
+          "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, rows 128 B
+// apart, groups of eight rows 1024 B apart (the layout a 128B-swizzled TMA box of
+// 32 fp32 x rows produces).  Tile bases are 1024-byte aligned.
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) |
+           (2ull << 61);
+}
+// Instruction descriptor: D = FP32, A = B = TF32, both K-major, M x N tile.
+__host__ __device__ constexpr uint32_t tc_idesc(int M, int N, bool negA) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((negA ? 1u : 0u) << 13) |
+           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+__global__ void __launch_bounds__(TC_THREADS, 1)
+cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                const TcParams p) {
+    extern __shared__ uint8_t tc_raw[];
+    const uint32_t raw_addr = smem_u32(tc_raw);
+    const uint32_t tiles = (raw_addr + 1023u) & ~1023u;             // stage buffers, 1024-aligned
+    uint8_t* ctl = tc_raw + (tiles - raw_addr) + TC_STAGES * TC_STAGE_BYTES;
+    const uint32_t bars = tiles + TC_STAGES * TC_STAGE_BYTES;
+    // barrier slots (8 bytes each): full[3] empty[3] tfull[2] tempty[2] drain
+    auto full = [&](int s) { return bars + 8u * s; };
+    auto empty = [&](int s) { return bars + 8u * (TC_STAGES + s); };
+    auto tfull = [&](int b) { return bars + 8u * (2 * TC_STAGES + b); };
+    auto tempty = [&](int b) { return bars + 8u * (2 * TC_STAGES + 2 + b); };
+    const uint32_t drain = bars + 8u * (2 * TC_STAGES + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + 128);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + 136);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), 128); }
+        mbar_init(drain, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(tmem_slot)), "r"(TC_TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int num_tiles = p.bins * p.m_tiles * p.n_tiles;
+    auto give_up = [&]() {
+        *abort_flag = 1;
+        if (p.status) atomicExch(p.status, 1);
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- producer ------------------------------------------------------
+            int it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; ok && t < num_tiles; t += gridDim.x) {
+                const int n_t = t % p.n_tiles;
+                const int m_t = (t / p.n_tiles) % p.m_tiles;
+                const int bin = t / (p.n_tiles * p.m_tiles);
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % TC_STAGES;
+                    const uint32_t ph = (uint32_t)(it / TC_STAGES) & 1u;
+                    if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t dst = tiles + s * TC_STAGE_BYTES;
+                    mbar_expect_tx(full(s), TC_STAGE_BYTES);
+                    tma_load_3d(dst + 0 * TC_TILE_BYTES, &tmA, kb * TC_BK, m_t * TC_BM, 2 * bin, full(s));
+                    tma_load_3d(dst + 1 * TC_TILE_BYTES, &tmA, kb * TC_BK, m_t * TC_BM, 2 * bin + 1, full(s));
+                    tma_load_3d(dst + 2 * TC_TILE_BYTES, &tmB, kb * TC_BK, n_t * TC_BN, 2 * bin, full(s));
+                    tma_load_3d(dst + 3 * TC_TILE_BYTES, &tmB, kb * TC_BK, n_t * TC_BN, 2 * bin + 1, full(s));
+                }
+            }
+            if (!ok) {
+                give_up();
+                // let the copies already issued land before the CTA's memory goes away
+                const int back = it < TC_STAGES ? it : TC_STAGES;
+                for (int j = it - back; j < it; ++j) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(full(j % TC_STAGES), (uint32_t)(j / TC_STAGES) & 1u) &&
+                           clock64() - t0 < TC_WAIT_CYCLES) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer ----------------------------------------------------
+            constexpr uint32_t idesc_pos = tc_idesc(TC_BM, TC_BN, false);
+            constexpr uint32_t idesc_neg = tc_idesc(TC_BM, TC_BN, true);
+            int it = 0, tl = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; ok && t < num_tiles; t += gridDim.x, ++tl) {
+                const int buf = tl & 1;
+                if (!mbar_wait(tempty(buf), ((uint32_t)(tl >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after_sync();
+                const uint32_t d_re = tmem_base + (uint32_t)buf * 256u;
+                const uint32_t d_im = d_re + 128u;
+                for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
+                    const int s = it % TC_STAGES;
+                    if (!mbar_wait(full(s), (uint32_t)(it / TC_STAGES) & 1u, abort_flag)) { ok = false; break; }
+                    tc_fence_after_sync();
+                    const uint32_t src = tiles + s * TC_STAGE_BYTES;
+                    const uint64_t a_re = tc_smem_desc(src), a_im = tc_smem_desc(src + TC_TILE_BYTES);
+                    const uint64_t b_re = tc_smem_desc(src + 2 * TC_TILE_BYTES);
+                    const uint64_t b_im = tc_smem_desc(src + 3 * TC_TILE_BYTES);
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 8; ++k) {
+                        const uint64_t adv = (uint64_t)(k * 2);        // 8 tf32 = 32 bytes = 2 x 16 B
+                        const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
+                        tc_mma_tf32(d_re, a_re + adv, b_re + adv, idesc_pos, acc);
+                        tc_mma_tf32(d_re, a_im + adv, b_im + adv, idesc_neg, 1u);
+                        tc_mma_tf32(d_im, a_re + adv, b_im + adv, idesc_pos, acc);
+                        tc_mma_tf32(d_im, a_im + adv, b_re + adv, idesc_pos, 1u);
+                    }
+                    tc_commit(empty(s));          // stage reusable once these MMAs have read it
+                }
+                if (ok) tc_commit(tfull(buf));    // accumulators complete
+            }
+            if (!ok) {
+                give_up();
+                tc_commit(drain);                 // wait (bounded) for the MMAs already issued
+                const long long t0 = clock64();
+                while (!mbar_try_wait(drain, 0u) && clock64() - t0 < TC_WAIT_CYCLES) {}
+            }
+        }
+    } else {
+        // ---- epilogue: warps 2..5, each owns the TMEM lanes of its quarter ------
+        const int q = warp & 3;
+        const size_t planeC = (size_t)p.M * p.ldc;
+        int tl = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; ok && t < num_tiles; t += gridDim.x, ++tl) {
+            const int n_t = t % p.n_tiles;
+            const int m_t = (t / p.n_tiles) % p.m_tiles;
+            const int bin = t / (p.n_tiles * p.m_tiles);
+            const int buf = tl & 1;
+            if (!mbar_wait(tfull(buf), (uint32_t)(tl >> 1) & 1u, abort_flag)) { ok = false; break; }
+            tc_fence_after_sync();
+            const int row = m_t * TC_BM + q * 32 + lane;
+            const int col0 = n_t * TC_BN;
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 256u;
+#pragma unroll 1
+            for (int part = 0; part < 2; ++part) {
+                float* out = p.C + ((size_t)bin * 2 + part) * planeC + (size_t)row * p.ldc + col0;
+#pragma unroll 1
+                for (int c = 0; c < TC_BN; c += 32) {
+                    if (col0 + c >= p.N) break;                     // warp-uniform
+                    uint32_t v[32];
+                    tc_ld32(t_row + (uint32_t)(part * 128 + c), v);
+                    tc_wait_ld();
+                    if (row < p.M) {
+                        if (col0 + c + 32 <= p.N) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<float4*>(out + c + j) =
+                                    make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + c + j < p.N) out[c + j] = __uint_as_float(v[j]);
+                        }
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(tempty(buf));
+        }
+        if (!ok && lane == 0) give_up();
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem_base), "r"(TC_TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side -------------------------------------------------------------
+typedef CUresult (*tc_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                 const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                 const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static tc_encode_fn tc_get_encode() {
+    static tc_encode_fn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) ==
+                cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<tc_encode_fn>(sym);
+    }
+    return fn;
+}
+
+// Planar operand [bins][2][rows][ld] seen as a 3-D tensor (k, row, bin*2+part);
+// out-of-range rows and k read as zero, which is what makes ragged M, N, K work.
+static bool tc_make_map(CUtensorMap* map, const float* base, int bins, int rows, int K, int ld,
+                        int box_rows) {
+    tc_encode_fn enc = tc_get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)bins * 2};
+    cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)rows * ld * 4};
+    cuuint32_t box[3] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides,
+               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static cudaError_t launch_cgemm_tc(const GemmParams& g, int* status, cudaStream_t st) {
+    static int sm_count = 0;
+    static bool attr_set = false;
+    if (!attr_set) {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(cgemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)TC_SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    CUtensorMap tmA, tmB;
+    if (!tc_make_map(&tmA, g.A, g.bins, g.M, g.K, g.lda, TC_BM)) return cudaErrorInvalidValue;
+    if (!tc_make_map(&tmB, g.B, g.bins, g.N, g.K, g.ldb, TC_BN)) return cudaErrorInvalidValue;
+    TcParams p{};
+    p.C = g.C; p.bins = g.bins; p.M = g.M; p.N = g.N; p.K = g.K; p.ldc = g.ldc;
+    p.m_tiles = (g.M + TC_BM - 1) / TC_BM;
+    p.n_tiles = (g.N + TC_BN - 1) / TC_BN;
+    p.k_blocks = (g.K + TC_BK - 1) / TC_BK;
+    p.status = status;
+    const long long tiles = (long long)p.bins * p.m_tiles * p.n_tiles;
+    if (tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
+    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+    cgemm_tc_kernel<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(tmA, tmB, p);
+    return cudaGetLastError();
+}
+
+}  // namespace fc
