@@ -137,16 +137,22 @@ int fft2d_c2r(const void* in_c, float* out, int batch, int n, int oh, int ow, fl
 
 /* Per-bin complex contraction alone (Table 1, the Cgemm row), exposed for
  * testing and profiling: for every bin b,
- *   C[b][m][nn] = sum_k A[b][m][k] * B[b][nn][k]         (no conjugation)
- * Operands are planar: A is device [bins][2][M][lda] fp32 (plane 0 real, plane
- * 1 imaginary, k contiguous, lda >= K), B likewise [bins][2][N][ldb], C
- * [bins][2][M][ldc] with ldc >= N.  lda, ldb, ldc must be multiples of 4.
+ *   C[b][m][nn] = sum_k op(A)[b][m][k] * op(B)[b][nn][k]
+ * with op = identity, or the complex conjugate when conjA / conjB is non-zero
+ * (Section 2: the conjugate turns the product into a cross-correlation).
+ * Operands are planar device arrays, plane 0 real and plane 1 imaginary:
+ *   A: [bins][2][M][lda], k contiguous (lda >= K); with transA != 0 it is stored
+ *      [bins][2][K][lda], m contiguous (lda >= M);
+ *   B: [bins][2][N][ldb] (ldb >= K), or with transB != 0 [bins][2][K][ldb] (ldb >= N);
+ *   C: [bins][2][M][ldc], ldc >= N; the padding columns N..ldc-1 are scratch
+ *      (they may be overwritten with zeros).
+ * lda, ldb, ldc must be multiples of 4 and the pointers 16-byte aligned.
  * math: FFTCONV_MATH_FP32 or FFTCONV_MATH_TF32 (AUTO resolves by shape).
- * status_word: device int the kernel sets non-zero if a bounded wait gives up;
- * may be NULL for the FP32 path. */
+ * status_word: device int the tensor-core kernel sets non-zero if a bounded wait
+ * gives up; may be NULL for the FP32 path. */
 int fftconv_bin_contract(const float* A, const float* B, float* C, int bins, int M, int N, int K,
-                         int lda, int ldb, int ldc, int math, int* status_word,
-                         void* cuda_stream);
+                         int lda, int ldb, int ldc, int transA, int transB, int conjA, int conjB,
+                         int math, int* status_word, void* cuda_stream);
 
 /* Text for a status code; never NULL. */
 const char* fftconv_status_string(int status);

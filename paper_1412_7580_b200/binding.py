@@ -57,7 +57,7 @@ def lib():
         L.conv_plan_stage_times_ms.argtypes = [p, p]
         L.fft2d_r2c.argtypes = [p, p, i, i, i, i, p]
         L.fft2d_c2r.argtypes = [p, p, i, i, i, i, fl, i, p]
-        L.fftconv_bin_contract.argtypes = [p, p, p] + [i] * 8 + [p, p]
+        L.fftconv_bin_contract.argtypes = [p, p, p] + [i] * 12 + [p, p]
         L.fftconv_status_string.argtypes = [i]
         L.fftconv_status_string.restype = ctypes.c_char_p
         L.fftconv_launch_count.argtypes = []
@@ -222,14 +222,17 @@ def fft2d_c2r(in_c, out, n, scale, accumulate=False, stream=None) -> None:
                            _stream_ptr(stream)), "fft2d_c2r")
 
 
-def fftconv_bin_contract(A, B, C, K, N=None, math=MATH_FP32, status_word=None, stream=None) -> None:
-    """A: [bins, 2, M, lda], B: [bins, 2, N, ldb], C: [bins, 2, M, ldc] float32 planar."""
-    bins, two, M, lda = A.shape
-    _, _, Nrows, ldb = B.shape
-    ldc = C.shape[3]
-    N = Nrows if N is None else N
+def fftconv_bin_contract(A, B, C, M, N, K, transA=False, transB=False, conjA=False, conjB=False,
+                         math=MATH_FP32, status_word=None, stream=None) -> None:
+    """Planar float32 operands: A [bins, 2, M, lda] (or [bins, 2, K, lda] with transA),
+    B [bins, 2, N, ldb] (or [bins, 2, K, ldb] with transB), C [bins, 2, M, ldc]."""
+    bins = A.shape[0]
+    assert A.shape[1] == 2 and B.shape[:2] == (bins, 2) and C.shape[:3] == (bins, 2, M)
+    assert A.shape[2] == (K if transA else M) and B.shape[2] == (K if transB else N)
+    lda, ldb, ldc = A.shape[3], B.shape[3], C.shape[3]
     sw = ctypes.c_void_p(status_word.data_ptr()) if status_word is not None else ctypes.c_void_p()
-    _check(lib().fftconv_bin_contract(_dev(A, None, "A"), _dev(B, (bins, 2, Nrows, ldb), "B"),
-                                      _dev(C, (bins, 2, M, ldc), "C"), bins, M, N, int(K),
-                                      lda, ldb, ldc, int(math), sw, _stream_ptr(stream)),
+    _check(lib().fftconv_bin_contract(_dev(A, None, "A"), _dev(B, None, "B"), _dev(C, None, "C"),
+                                      bins, int(M), int(N), int(K), lda, ldb, ldc,
+                                      int(bool(transA)), int(bool(transB)), int(bool(conjA)),
+                                      int(bool(conjB)), int(math), sw, _stream_ptr(stream)),
            "fftconv_bin_contract")

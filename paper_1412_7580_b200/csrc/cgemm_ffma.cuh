@@ -1,9 +1,10 @@
 // Per-frequency-bin complex contraction with FP32 FFMA (Table 1, the Cgemm row).
 //
-// For every bin b:  C[b][m][n] = sum_k A[b][m][k] * B[b][n][k]   (complex, no
-// conjugation -- conjugates were folded into the forward FFT's store).
-// Operands are planar and k-contiguous: A is [bins][2][M][lda] (plane 0 real,
-// plane 1 imaginary), B is [bins][2][N][ldb], C is [bins][2][M][ldc].
+// For every bin b:  C[b][m][n] = sum_k op(A)[b][m][k] * op(B)[b][n][k]  (complex;
+// op = identity or complex conjugate).
+// Operands are planar (plane 0 real, plane 1 imaginary).  A is [bins][2][M][lda]
+// (k contiguous) or, with transA, [bins][2][K][lda] (m contiguous); B likewise
+// [bins][2][N][ldb] or, with transB, [bins][2][K][ldb]; C is [bins][2][M][ldc].
 //
 // CTA tile 64 x 64 of one bin, 256 threads, each thread a 4 x 4 block of complex
 // outputs (64 FFMAs per k against four 16-byte shared loads).  This is the exact
@@ -20,6 +21,8 @@ struct GemmParams {
     float* C;
     int bins, M, N, K;
     int lda, ldb, ldc;
+    int transA, transB;   // operand stored [K][rows] instead of [rows][K]
+    int conjA, conjB;     // use the complex conjugate of the operand
 };
 
 constexpr int FG_BM = 64, FG_BN = 64, FG_BK = 16, FG_PAD = 4, FG_T = 256;
@@ -31,8 +34,9 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
     const int tid = threadIdx.x;
     const int bin = blockIdx.z;
     const int m_blk = blockIdx.y * FG_BM, n_blk = blockIdx.x * FG_BN;
-    const size_t planeA = (size_t)p.M * p.lda, planeB = (size_t)p.N * p.ldb,
-                 planeC = (size_t)p.M * p.ldc;
+    const size_t planeA = (size_t)(p.transA ? p.K : p.M) * p.lda,
+                 planeB = (size_t)(p.transB ? p.K : p.N) * p.ldb, planeC = (size_t)p.M * p.ldc;
+    const float sa = p.conjA ? -1.0f : 1.0f, sb = p.conjB ? -1.0f : 1.0f;
     const float* Ab = p.A + (size_t)bin * 2 * planeA;
     const float* Bb = p.B + (size_t)bin * 2 * planeB;
     float* Cb = p.C + (size_t)bin * 2 * planeC;
@@ -47,24 +51,57 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
         for (int j = 0; j < 4; ++j) cr[i][j] = ci[i][j] = 0.0f;
 
     for (int k0 = 0; k0 < p.K; k0 += FG_BK) {
-        // global -> shared, transposing to [k][row]; zero-fill outside M/N/K
-        const int k = k0 + lk;
-        const bool kin = k < p.K;
+        // global -> shared as [k][row]; zero-fill outside M/N/K; lanes run along the
+        // contiguous index of each operand
+        if (!p.transA) {
+            const int k = k0 + lk;
 #pragma unroll
-        for (int it = 0; it < FG_BM / 16; ++it) {
-            const int r = lr + 16 * it;
-            const int m = m_blk + r, n = n_blk + r;
-            float are = 0.f, aim = 0.f, bre = 0.f, bim = 0.f;
-            if (kin && m < p.M) {
-                are = __ldg(Ab + (size_t)m * p.lda + k);
-                aim = __ldg(Ab + planeA + (size_t)m * p.lda + k);
+            for (int it = 0; it < FG_BM / 16; ++it) {
+                const int r = lr + 16 * it, m = m_blk + r;
+                float are = 0.f, aim = 0.f;
+                if (k < p.K && m < p.M) {
+                    are = __ldg(Ab + (size_t)m * p.lda + k);
+                    aim = sa * __ldg(Ab + planeA + (size_t)m * p.lda + k);
+                }
+                sA[0][lk][r] = are; sA[1][lk][r] = aim;
             }
-            if (kin && n < p.N) {
-                bre = __ldg(Bb + (size_t)n * p.ldb + k);
-                bim = __ldg(Bb + planeB + (size_t)n * p.ldb + k);
+        } else {
+            const int r = tid & 63, m = m_blk + r;
+#pragma unroll
+            for (int it = 0; it < FG_BK / 4; ++it) {
+                const int kk = (tid >> 6) + 4 * it, k = k0 + kk;
+                float are = 0.f, aim = 0.f;
+                if (k < p.K && m < p.M) {
+                    are = __ldg(Ab + (size_t)k * p.lda + m);
+                    aim = sa * __ldg(Ab + planeA + (size_t)k * p.lda + m);
+                }
+                sA[0][kk][r] = are; sA[1][kk][r] = aim;
             }
-            sA[0][lk][r] = are; sA[1][lk][r] = aim;
-            sB[0][lk][r] = bre; sB[1][lk][r] = bim;
+        }
+        if (!p.transB) {
+            const int k = k0 + lk;
+#pragma unroll
+            for (int it = 0; it < FG_BN / 16; ++it) {
+                const int r = lr + 16 * it, n = n_blk + r;
+                float bre = 0.f, bim = 0.f;
+                if (k < p.K && n < p.N) {
+                    bre = __ldg(Bb + (size_t)n * p.ldb + k);
+                    bim = sb * __ldg(Bb + planeB + (size_t)n * p.ldb + k);
+                }
+                sB[0][lk][r] = bre; sB[1][lk][r] = bim;
+            }
+        } else {
+            const int r = tid & 63, n = n_blk + r;
+#pragma unroll
+            for (int it = 0; it < FG_BK / 4; ++it) {
+                const int kk = (tid >> 6) + 4 * it, k = k0 + kk;
+                float bre = 0.f, bim = 0.f;
+                if (k < p.K && n < p.N) {
+                    bre = __ldg(Bb + (size_t)k * p.ldb + n);
+                    bim = sb * __ldg(Bb + planeB + (size_t)k * p.ldb + n);
+                }
+                sB[0][kk][r] = bre; sB[1][kk][r] = bim;
+            }
         }
         __syncthreads();
 #pragma unroll

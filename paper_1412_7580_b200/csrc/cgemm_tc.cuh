@@ -1,7 +1,11 @@
 // Per-frequency-bin complex contraction on the 5th-generation tensor cores
 // (Table 1, the Cgemm row): for every bin b,
-//     C[b][m][n] = sum_k A[b][m][k] * B[b][n][k]          (complex)
-// with planar, k-contiguous operands (see cgemm_ffma.cuh for the layout).
+//     C[b][m][n] = sum_k op(A)[b][m][k] * op(B)[b][n][k]      (complex)
+// with planar operands (see cgemm_ffma.cuh for the layouts): each operand is
+// stored either k-contiguous ([rows][k]) or row-contiguous ([k][rows]); the
+// second form is fed to the tensor cores as an "MN-major" shared-memory matrix,
+// so no pass ever needs a transposed copy of a spectrum.  op() is an optional
+// complex conjugate, folded into the negate bits below.
 //
 // The complex product is four real TF32 MMAs per k-step into two FP32
 // accumulators in tensor memory,
@@ -13,9 +17,11 @@
 //   warp 0      TMA producer: 128-byte-swizzled boxes of 32 k-values x 128 rows
 //               of A_re, A_im, B_re, B_im per stage (64 KB), 3 stages in flight;
 //   warp 1      issues tcgen05.mma (one lane), owns the TMEM allocation;
-//   warps 2..5  epilogue: tcgen05.ld of the finished accumulators and stores to
-//               the frequency-major result, overlapped with the next tile's MMAs
-//               through two accumulator buffers (2 x 256 TMEM columns).
+//   warps 2..5  epilogue: tcgen05.ld of the finished accumulators, a swizzled
+//               staging tile per warp in shared memory and TMA stores (full
+//               128-byte lines, clipped at the matrix edge by the tensor map),
+//               overlapped with the next tile's MMAs through two accumulator
+//               buffers (2 x 256 TMEM columns).
 // The per-bin problems are small and the kernel streams: it is bound by HBM
 // bytes (two spectra in, one out), not by tensor throughput.
 //
@@ -36,14 +42,16 @@ constexpr int TC_BM = 128, TC_BN = 128, TC_BK = 32, TC_STAGES = 3;
 constexpr int TC_THREADS = 192;
 constexpr uint32_t TC_TILE_BYTES = TC_BM * TC_BK * 4;            // one 128 x 32 fp32 box: 16 KB
 constexpr uint32_t TC_STAGE_BYTES = 4 * TC_TILE_BYTES;           // A_re, A_im, B_re, B_im
-constexpr uint32_t TC_SMEM_BYTES = 1024 + TC_STAGES * TC_STAGE_BYTES + 256;
+constexpr uint32_t TC_EPI_BUF_BYTES = 32 * 128;                  // 32 rows x 32 fp32, one TMA store box
+constexpr uint32_t TC_EPI_BYTES = 4 * 2 * TC_EPI_BUF_BYTES;      // 4 warps x 2 buffers
+constexpr uint32_t TC_SMEM_BYTES = 1024 + TC_STAGES * TC_STAGE_BYTES + TC_EPI_BYTES + 256;
 constexpr uint32_t TC_TMEM_COLS = 512;
 constexpr long long TC_WAIT_CYCLES = 2000000000LL;               // about one second
 
 struct TcParams {
-    float* C;
-    int bins, M, N, K, ldc;
+    int bins, M, N, K;
     int m_tiles, n_tiles, k_blocks;
+    int conjA, conjB;
     int* status;
 };
 
@@ -97,6 +105,13 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1,
+                                             int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
 __device__ __forceinline__ void tc_fence_before_sync() {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -140,20 +155,34 @@ __device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr) {
     return (uint64_t)((saddr >> 4) & 0x3FFF) | (1ull << 16) | (64ull << 32) | (1ull << 46) |
            (2ull << 61);
 }
-// Instruction descriptor: D = FP32, A = B = TF32, both K-major, M x N tile.
-__host__ __device__ constexpr uint32_t tc_idesc(int M, int N, bool negA) {
+// MN-major TF32 operand: the only shared-memory layout the tensor cores take for
+// it is the 128-byte swizzle with a 32-byte base (32-byte chunks of a 128-byte
+// row are permuted by the row index modulo 4), which the TMA produces with its
+// "128B, 32B atom" mode.  The tile is four blocks of 32 rows-of-the-matrix
+// (128 B, contiguous in memory) x 32 k; inside a block consecutive k are 128 B
+// apart, groups of four k 512 B apart (stride offset); blocks are 4096 B apart
+// (leading offset).  One MMA consumes eight k = 1024 bytes.
+__device__ __forceinline__ uint64_t tc_smem_desc_mn(uint32_t saddr) {
+    return (uint64_t)((saddr >> 4) & 0x3FFF) | (256ull << 16) | (32ull << 32) | (1ull << 46) |
+           (1ull << 61);
+}
+// Instruction descriptor: D = FP32, A = B = TF32, M x N tile; majorness per operand.
+__host__ __device__ constexpr uint32_t tc_idesc(int M, int N, bool negA, bool mnA, bool mnB) {
     return (1u << 4) | (2u << 7) | (2u << 10) | ((negA ? 1u : 0u) << 13) |
+           ((mnA ? 1u : 0u) << 15) | ((mnB ? 1u : 0u) << 16) |
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
+template <bool TA, bool TB>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                const TcParams p) {
+                const __grid_constant__ CUtensorMap tmC, const TcParams p) {
     extern __shared__ uint8_t tc_raw[];
     const uint32_t raw_addr = smem_u32(tc_raw);
     const uint32_t tiles = (raw_addr + 1023u) & ~1023u;             // stage buffers, 1024-aligned
-    uint8_t* ctl = tc_raw + (tiles - raw_addr) + TC_STAGES * TC_STAGE_BYTES;
-    const uint32_t bars = tiles + TC_STAGES * TC_STAGE_BYTES;
+    const uint32_t epi = tiles + TC_STAGES * TC_STAGE_BYTES;        // epilogue staging, 1024-aligned
+    uint8_t* ctl = tc_raw + (tiles - raw_addr) + TC_STAGES * TC_STAGE_BYTES + TC_EPI_BYTES;
+    const uint32_t bars = epi + TC_EPI_BYTES;
     // barrier slots (8 bytes each): full[3] empty[3] tfull[2] tempty[2] drain
     auto full = [&](int s) { return bars + 8u * s; };
     auto empty = [&](int s) { return bars + 8u * (TC_STAGES + s); };
@@ -203,10 +232,27 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t dst = tiles + s * TC_STAGE_BYTES;
                     mbar_expect_tx(full(s), TC_STAGE_BYTES);
-                    tma_load_3d(dst + 0 * TC_TILE_BYTES, &tmA, kb * TC_BK, m_t * TC_BM, 2 * bin, full(s));
-                    tma_load_3d(dst + 1 * TC_TILE_BYTES, &tmA, kb * TC_BK, m_t * TC_BM, 2 * bin + 1, full(s));
-                    tma_load_3d(dst + 2 * TC_TILE_BYTES, &tmB, kb * TC_BK, n_t * TC_BN, 2 * bin, full(s));
-                    tma_load_3d(dst + 3 * TC_TILE_BYTES, &tmB, kb * TC_BK, n_t * TC_BN, 2 * bin + 1, full(s));
+#pragma unroll
+                    for (int part = 0; part < 2; ++part) {
+                        if constexpr (!TA) {
+                            tma_load_3d(dst + part * TC_TILE_BYTES, &tmA, kb * TC_BK, m_t * TC_BM,
+                                        2 * bin + part, full(s));
+                        } else {
+#pragma unroll
+                            for (int blk = 0; blk < 4; ++blk)
+                                tma_load_3d(dst + part * TC_TILE_BYTES + blk * 4096, &tmA,
+                                            m_t * TC_BM + blk * 32, kb * TC_BK, 2 * bin + part, full(s));
+                        }
+                        if constexpr (!TB) {
+                            tma_load_3d(dst + (2 + part) * TC_TILE_BYTES, &tmB, kb * TC_BK, n_t * TC_BN,
+                                        2 * bin + part, full(s));
+                        } else {
+#pragma unroll
+                            for (int blk = 0; blk < 4; ++blk)
+                                tma_load_3d(dst + (2 + part) * TC_TILE_BYTES + blk * 4096, &tmB,
+                                            n_t * TC_BN + blk * 32, kb * TC_BK, 2 * bin + part, full(s));
+                        }
+                    }
                 }
             }
             if (!ok) {
@@ -223,8 +269,12 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     } else if (warp == 1) {
         if (lane == 0) {
             // ---- MMA issuer ----------------------------------------------------
-            constexpr uint32_t idesc_pos = tc_idesc(TC_BM, TC_BN, false);
-            constexpr uint32_t idesc_neg = tc_idesc(TC_BM, TC_BN, true);
+            constexpr uint32_t idesc_pos = tc_idesc(TC_BM, TC_BN, false, TA, TB);
+            constexpr uint32_t idesc_neg = tc_idesc(TC_BM, TC_BN, true, TA, TB);
+            // (Ar + i sA Ai)(Br + i sB Bi): re = ArBr - sA sB AiBi ; im = sB ArBi + sA AiBr
+            const uint32_t id_ii = (p.conjA != p.conjB) ? idesc_pos : idesc_neg;
+            const uint32_t id_ri = p.conjB ? idesc_neg : idesc_pos;
+            const uint32_t id_ir = p.conjA ? idesc_neg : idesc_pos;
             int it = 0, tl = 0;
             bool ok = true;
             for (int t = blockIdx.x; ok && t < num_tiles; t += gridDim.x, ++tl) {
@@ -238,17 +288,24 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     if (!mbar_wait(full(s), (uint32_t)(it / TC_STAGES) & 1u, abort_flag)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t src = tiles + s * TC_STAGE_BYTES;
-                    const uint64_t a_re = tc_smem_desc(src), a_im = tc_smem_desc(src + TC_TILE_BYTES);
-                    const uint64_t b_re = tc_smem_desc(src + 2 * TC_TILE_BYTES);
-                    const uint64_t b_im = tc_smem_desc(src + 3 * TC_TILE_BYTES);
+                    const uint64_t a_re = TA ? tc_smem_desc_mn(src) : tc_smem_desc(src);
+                    const uint64_t a_im = TA ? tc_smem_desc_mn(src + TC_TILE_BYTES)
+                                             : tc_smem_desc(src + TC_TILE_BYTES);
+                    const uint64_t b_re = TB ? tc_smem_desc_mn(src + 2 * TC_TILE_BYTES)
+                                             : tc_smem_desc(src + 2 * TC_TILE_BYTES);
+                    const uint64_t b_im = TB ? tc_smem_desc_mn(src + 3 * TC_TILE_BYTES)
+                                             : tc_smem_desc(src + 3 * TC_TILE_BYTES);
+                    // per k-step of 8: K-major advances 32 bytes inside the swizzled row,
+                    // MN-major advances eight 128-byte k-rows (address field is in 16 B units)
+                    constexpr uint64_t stepA = TA ? 64 : 2, stepB = TB ? 64 : 2;
 #pragma unroll
                     for (int k = 0; k < TC_BK / 8; ++k) {
-                        const uint64_t adv = (uint64_t)(k * 2);        // 8 tf32 = 32 bytes = 2 x 16 B
+                        const uint64_t da = stepA * k, db = stepB * k;
                         const uint32_t acc = (kb | k) != 0 ? 1u : 0u;
-                        tc_mma_tf32(d_re, a_re + adv, b_re + adv, idesc_pos, acc);
-                        tc_mma_tf32(d_re, a_im + adv, b_im + adv, idesc_neg, 1u);
-                        tc_mma_tf32(d_im, a_re + adv, b_im + adv, idesc_pos, acc);
-                        tc_mma_tf32(d_im, a_im + adv, b_re + adv, idesc_pos, 1u);
+                        tc_mma_tf32(d_re, a_re + da, b_re + db, idesc_pos, acc);
+                        tc_mma_tf32(d_re, a_im + da, b_im + db, id_ii, 1u);
+                        tc_mma_tf32(d_im, a_re + da, b_im + db, id_ri, acc);
+                        tc_mma_tf32(d_im, a_im + da, b_re + db, id_ir, 1u);
                     }
                     tc_commit(empty(s));          // stage reusable once these MMAs have read it
                 }
@@ -264,8 +321,9 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     } else {
         // ---- epilogue: warps 2..5, each owns the TMEM lanes of its quarter ------
         const int q = warp & 3;
-        const size_t planeC = (size_t)p.M * p.ldc;
+        const uint32_t my_buf = epi + (uint32_t)q * 2u * TC_EPI_BUF_BYTES;
         int tl = 0;
+        uint32_t nstore = 0;
         bool ok = true;
         for (int t = blockIdx.x; ok && t < num_tiles; t += gridDim.x, ++tl) {
             const int n_t = t % p.n_tiles;
@@ -274,36 +332,45 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int buf = tl & 1;
             if (!mbar_wait(tfull(buf), (uint32_t)(tl >> 1) & 1u, abort_flag)) { ok = false; break; }
             tc_fence_after_sync();
-            const int row = m_t * TC_BM + q * 32 + lane;
+            const int row0 = m_t * TC_BM + q * 32;
             const int col0 = n_t * TC_BN;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)buf * 256u;
+            if (row0 < p.M) {                                           // warp-uniform
 #pragma unroll 1
-            for (int part = 0; part < 2; ++part) {
-                float* out = p.C + ((size_t)bin * 2 + part) * planeC + (size_t)row * p.ldc + col0;
+                for (int part = 0; part < 2; ++part) {
 #pragma unroll 1
-                for (int c = 0; c < TC_BN; c += 32) {
-                    if (col0 + c >= p.N) break;                     // warp-uniform
-                    uint32_t v[32];
-                    tc_ld32(t_row + (uint32_t)(part * 128 + c), v);
-                    tc_wait_ld();
-                    if (row < p.M) {
-                        if (col0 + c + 32 <= p.N) {
+                    for (int c = 0; c < TC_BN; c += 32) {
+                        if (col0 + c >= p.N) break;                     // warp-uniform
+                        uint32_t v[32];
+                        tc_ld32(t_row + (uint32_t)(part * 128 + c), v);
+                        // the staging buffer used two stores ago must have been read out
+                        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        __syncwarp();
+                        tc_wait_ld();
+                        // row = lane; 16-byte chunk j goes to slot j ^ (row % 8) (128-byte swizzle)
+                        const uint32_t sbuf = my_buf + (nstore & 1u) * TC_EPI_BUF_BYTES;
+                        const uint32_t srow = sbuf + (uint32_t)lane * 128u;
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<float4*>(out + c + j) =
-                                    make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
-                                                __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + c + j < p.N) out[c + j] = __uint_as_float(v[j]);
+                        for (int j = 0; j < 8; ++j)
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                                         ::"r"(srow + (uint32_t)((j ^ (lane & 7)) << 4)), "r"(v[4 * j]),
+                                           "r"(v[4 * j + 1]), "r"(v[4 * j + 2]), "r"(v[4 * j + 3])
+                                         : "memory");
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        __syncwarp();
+                        if (lane == 0) {
+                            tma_store_3d(&tmC, sbuf, col0 + c, row0, 2 * bin + part);
+                            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                         }
+                        ++nstore;
                     }
                 }
             }
             tc_fence_before_sync();
             mbar_arrive(tempty(buf));
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+        __syncwarp();
         if (!ok && lane == 0) give_up();
     }
 
@@ -336,49 +403,71 @@ static tc_encode_fn tc_get_encode() {
     return fn;
 }
 
-// Planar operand [bins][2][rows][ld] seen as a 3-D tensor (k, row, bin*2+part);
-// out-of-range rows and k read as zero, which is what makes ragged M, N, K work.
-static bool tc_make_map(CUtensorMap* map, const float* base, int bins, int rows, int K, int ld,
-                        int box_rows) {
+// Planar matrix family [bins][2][rows][ld] seen as a 3-D tensor (col, row,
+// bin*2+part) with `cols` valid columns; out-of-range coordinates read as zero
+// and are clipped on store, which is what makes ragged M, N, K work.
+static bool tc_make_map(CUtensorMap* map, const float* base, int bins, int rows, int cols, int ld,
+                        int box_cols, int box_rows,
+                        CUtensorMapSwizzle swz = CU_TENSOR_MAP_SWIZZLE_128B) {
     tc_encode_fn enc = tc_get_encode();
     if (!enc) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)bins * 2};
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)bins * 2};
     cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)rows * ld * 4};
-    cuuint32_t box[3] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows, 1};
+    cuuint32_t box[3] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1};
     cuuint32_t estr[3] = {1, 1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides,
-               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool TA, bool TB>
+static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStream_t st, int sm_count) {
+    auto kern = cgemm_tc_kernel<TA, TB>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)TC_SMEM_BYTES);
+        if (e != cudaSuccess) return e;
+        attr_set = true;
+    }
+    CUtensorMap tmA, tmB, tmC;
+    // k-contiguous: rows = M (or N), cols = K, box 32 k x 128 rows;
+    // row-contiguous: rows = K, cols = M (or N), box 32 rows-of-the-matrix x 32 k.
+    const bool okA = TA ? tc_make_map(&tmA, g.A, g.bins, g.K, g.M, g.lda, 32, TC_BK,
+                                      CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)
+                        : tc_make_map(&tmA, g.A, g.bins, g.M, g.K, g.lda, TC_BK, TC_BM);
+    const bool okB = TB ? tc_make_map(&tmB, g.B, g.bins, g.K, g.N, g.ldb, 32, TC_BK,
+                                      CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)
+                        : tc_make_map(&tmB, g.B, g.bins, g.N, g.K, g.ldb, TC_BK, TC_BN);
+    const bool okC = tc_make_map(&tmC, g.C, g.bins, g.M, g.N, g.ldc, 32, 32);
+    if (!okA || !okB || !okC) return cudaErrorInvalidValue;
+    TcParams p{};
+    p.bins = g.bins; p.M = g.M; p.N = g.N; p.K = g.K;
+    p.m_tiles = (g.M + TC_BM - 1) / TC_BM;
+    p.n_tiles = (g.N + TC_BN - 1) / TC_BN;
+    p.k_blocks = (g.K + TC_BK - 1) / TC_BK;
+    p.conjA = g.conjA; p.conjB = g.conjB;
+    p.status = status;
+    const long long tiles = (long long)p.bins * p.m_tiles * p.n_tiles;
+    if (tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
+    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
+    kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(tmA, tmB, tmC, p);
+    return cudaGetLastError();
 }
 
 static cudaError_t launch_cgemm_tc(const GemmParams& g, int* status, cudaStream_t st) {
     static int sm_count = 0;
-    static bool attr_set = false;
-    if (!attr_set) {
+    if (sm_count == 0) {
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
         if (e != cudaSuccess) return e;
         e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
         if (e != cudaSuccess) return e;
-        e = cudaFuncSetAttribute(cgemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)TC_SMEM_BYTES);
-        if (e != cudaSuccess) return e;
-        attr_set = true;
     }
-    CUtensorMap tmA, tmB;
-    if (!tc_make_map(&tmA, g.A, g.bins, g.M, g.K, g.lda, TC_BM)) return cudaErrorInvalidValue;
-    if (!tc_make_map(&tmB, g.B, g.bins, g.N, g.K, g.ldb, TC_BN)) return cudaErrorInvalidValue;
-    TcParams p{};
-    p.C = g.C; p.bins = g.bins; p.M = g.M; p.N = g.N; p.K = g.K; p.ldc = g.ldc;
-    p.m_tiles = (g.M + TC_BM - 1) / TC_BM;
-    p.n_tiles = (g.N + TC_BN - 1) / TC_BN;
-    p.k_blocks = (g.K + TC_BK - 1) / TC_BK;
-    p.status = status;
-    const long long tiles = (long long)p.bins * p.m_tiles * p.n_tiles;
-    if (tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
-    const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    cgemm_tc_kernel<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(tmA, tmB, p);
-    return cudaGetLastError();
+    if (g.transA) return g.transB ? launch_cgemm_tc_t<true, true>(g, status, st, sm_count)
+                                  : launch_cgemm_tc_t<true, false>(g, status, st, sm_count);
+    return g.transB ? launch_cgemm_tc_t<false, true>(g, status, st, sm_count)
+                    : launch_cgemm_tc_t<false, false>(g, status, st, sm_count);
 }
 
 }  // namespace fc

@@ -33,18 +33,17 @@ struct SpecDesc {
     size_t bytes(int bins) const { return (size_t)bins * 2 * R * ld * sizeof(float); }
 };
 
-// How one real tensor enters a pass: plane p of the BDHW tensor goes to matrix
-// position (row, col) with p = row*in_rs + col*in_cs.
+// One real tensor of a pass and its spectrum: plane (row, col) of the BDHW tensor
+// is matrix element (row, col) of every bin.
 struct OperandDesc {
     SpecDesc spec;
     int h, w;               // plane size (forward) or crop window (inverse)
-    long long in_rs, in_cs;
-    int conj;
 };
 
 struct PassDesc {
     OperandDesc a, b, c;    // c: result (h, w = crop window)
-    int M, N, K;            // per-bin contraction C[M][N] = sum_K A[M][K] B[N][K]
+    int M, N, K;            // per-bin contraction C[M][N] = sum_K op(A)[M][K] op(B)[N][K]
+    int transA, transB, conjA, conjB;
 };
 
 enum { PASS_FPROP = 0, PASS_BPROP = 1, PASS_ACCGRAD = 2 };
@@ -66,31 +65,34 @@ struct conv_plan_s {
 namespace {
 
 // Operand roles per pass (Table 1 and Section 2; which operand carries the
-// conjugate follows from the convolution theorem for cross-correlation):
-//   fprop  : X^[b][s][i] , conj W^[b][j][i] -> Y^[b][s][j]     reduce over f
-//   bprop  : dY^[b][s][j],      W^[b][i][j] -> dX^[b][s][i]    reduce over f'
-//   accGrad: conj dY^[b][j][s], X^[b][i][s] -> dW^[b][j][i]    reduce over S
+// conjugate follows from the convolution theorem for cross-correlation).  Every
+// spectrum keeps the plane order of its tensor ([S][f], [f'][f], [S][f']); where
+// the summed index is not the minor one the contraction reads the operand
+// "transposed" ([k][rows]) instead of the FFT writing a transposed copy.
+//   fprop  : Y^[b][s][j]  = sum_i X^[b][s][i]        conj W^[b][j][i]
+//   bprop  : dX^[b][s][i] = sum_j dY^[b][s][j]       W^[b][j][i]        (B read as [k=j][i])
+//   accGrad: dW^[b][j][i] = sum_s conj dY^[b][s][j]  X^[b][s][i]        (A as [k=s][j], B as [k=s][i])
 PassDesc describe(const conv_plan_s& p, int pass) {
     PassDesc d{};
     auto spec = [](int R, int C) { return SpecDesc{R, C, round4(C)}; };
+    const OperandDesc X = {spec(p.S, p.f), p.h, p.w};
+    const OperandDesc W = {spec(p.fp, p.f), p.kh, p.kw};
+    const OperandDesc Y = {spec(p.S, p.fp), p.oh, p.ow};
     switch (pass) {
         case PASS_FPROP:
-            d.a = {spec(p.S, p.f), p.h, p.w, p.f, 1, 0};
-            d.b = {spec(p.fp, p.f), p.kh, p.kw, p.f, 1, 1};
-            d.c = {spec(p.S, p.fp), p.oh, p.ow, 0, 0, 0};
+            d.a = X; d.b = W; d.c = Y;
             d.M = p.S; d.N = p.fp; d.K = p.f;
+            d.transA = 0; d.transB = 0; d.conjA = 0; d.conjB = 1;
             break;
         case PASS_BPROP:
-            d.a = {spec(p.S, p.fp), p.oh, p.ow, p.fp, 1, 0};
-            d.b = {spec(p.f, p.fp), p.kh, p.kw, 1, p.f, 0};      // w[j][i] -> row i, col j
-            d.c = {spec(p.S, p.f), p.h, p.w, 0, 0, 0};
+            d.a = Y; d.b = W; d.c = X;
             d.M = p.S; d.N = p.f; d.K = p.fp;
+            d.transA = 0; d.transB = 1; d.conjA = 0; d.conjB = 0;
             break;
         default:
-            d.a = {spec(p.fp, p.S), p.oh, p.ow, 1, p.fp, 1};     // dy[s][j] -> row j, col s
-            d.b = {spec(p.f, p.S), p.h, p.w, 1, p.f, 0};         // x[s][i]  -> row i, col s
-            d.c = {spec(p.fp, p.f), p.kh, p.kw, 0, 0, 0};
+            d.a = Y; d.b = X; d.c = W;
             d.M = p.fp; d.N = p.f; d.K = p.S;
+            d.transA = 1; d.transB = 1; d.conjA = 1; d.conjB = 0;
             break;
     }
     return d;
@@ -129,7 +131,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         fp.real_in = in; fp.spec_out = spec;
         fp.h = o.h; fp.w = o.w;
         fp.R = o.spec.R; fp.C = o.spec.C; fp.ld = o.spec.ld;
-        fp.in_rs = o.in_rs; fp.in_cs = o.in_cs; fp.conj = o.conj;
+        fp.in_rs = o.spec.C; fp.in_cs = 1; fp.conj = 0;
         g_launches.fetch_add(1, std::memory_order_relaxed);
         return fc::launch_r2c<fc::LAYOUT_FREQ_MAJOR>(plan->n, fp, st);
     };
@@ -145,6 +147,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     gp.A = specA; gp.B = specB; gp.C = specC;
     gp.bins = plan->bins; gp.M = d.M; gp.N = d.N; gp.K = d.K;
     gp.lda = d.a.spec.ld; gp.ldb = d.b.spec.ld; gp.ldc = d.c.spec.ld;
+    gp.transA = d.transA; gp.transB = d.transB; gp.conjA = d.conjA; gp.conjB = d.conjB;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     cudaError_t ge;
     if (resolve_math(*plan, d) == FFTCONV_MATH_TF32) ge = fc::launch_cgemm_tc(gp, status, st);
@@ -320,10 +323,13 @@ FFTCONV_API int fft2d_c2r(const void* in_c, float* out, int batch, int n, int oh
 }
 
 FFTCONV_API int fftconv_bin_contract(const float* A, const float* B, float* C, int bins, int M,
-                                     int N, int K, int lda, int ldb, int ldc, int math,
+                                     int N, int K, int lda, int ldb, int ldc, int transA,
+                                     int transB, int conjA, int conjB, int math,
                                      int* status_word, void* cuda_stream) {
     if (!A || !B || !C || bins < 1 || M < 1 || N < 1 || K < 1) return FFTCONV_EINVAL;
-    if (lda < K || ldb < K || ldc < N || (lda & 3) || (ldb & 3) || (ldc & 3)) return FFTCONV_EINVAL;
+    if (lda < (transA ? M : K) || ldb < (transB ? N : K) || ldc < N || (lda & 3) || (ldb & 3) ||
+        (ldc & 3))
+        return FFTCONV_EINVAL;
     if (((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(B) |
           reinterpret_cast<uintptr_t>(C)) & 15) != 0)
         return FFTCONV_EINVAL;
@@ -332,6 +338,8 @@ FFTCONV_API int fftconv_bin_contract(const float* A, const float* B, float* C, i
     gp.A = A; gp.B = B; gp.C = C;
     gp.bins = bins; gp.M = M; gp.N = N; gp.K = K;
     gp.lda = lda; gp.ldb = ldb; gp.ldc = ldc;
+    gp.transA = transA ? 1 : 0; gp.transB = transB ? 1 : 0;
+    gp.conjA = conjA ? 1 : 0; gp.conjB = conjB ? 1 : 0;
     int eff = math;
     if (math == FFTCONV_MATH_AUTO)
         eff = (fc::tc_shape_supported(M, N, K) && fc::tc_shape_profitable(M, N, K))

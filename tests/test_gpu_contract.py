@@ -8,35 +8,44 @@ pytestmark = pytest.mark.gpu
 TOL = {1: 1e-4, 2: 5e-3}
 
 
-def run(bins, M, N, K, math, seed=0):
+def run(bins, M, N, K, math, seed=0, transA=False, transB=False, conjA=False, conjB=False):
     import torch
     import oracle
     import paper_1412_7580_b200 as fc
     rng = np.random.default_rng([14127580, 55, seed, bins, M, N, K])
-    lda = ldb = (K + 3) // 4 * 4
-    ldc = (N + 3) // 4 * 4
-    A = np.zeros((bins, 2, M, lda), np.float32)
-    B = np.zeros((bins, 2, N, ldb), np.float32)
-    A[..., :K] = rng.standard_normal((bins, 2, M, K), dtype=np.float32)
-    B[..., :K] = rng.standard_normal((bins, 2, N, K), dtype=np.float32)
-    # padding columns hold garbage that must never be read as data
-    A[..., K:] = 1e30
-    B[..., K:] = -1e30
+    r4 = lambda v: (v + 3) // 4 * 4
+
+    def operand(rows, trans, fill):
+        """Logical [bins][rows][K] complex matrix, stored planar either as
+        [bins][2][rows][ld>=K] or, transposed, as [bins][2][K][ld>=rows]."""
+        re = rng.standard_normal((bins, rows, K), dtype=np.float32)
+        im = rng.standard_normal((bins, rows, K), dtype=np.float32)
+        if not trans:
+            buf = np.full((bins, 2, rows, r4(K)), fill, np.float32)   # padding must never be read as data
+            buf[:, 0, :, :K], buf[:, 1, :, :K] = re, im
+        else:
+            buf = np.full((bins, 2, K, r4(rows)), fill, np.float32)
+            buf[:, 0, :, :rows], buf[:, 1, :, :rows] = re.transpose(0, 2, 1), im.transpose(0, 2, 1)
+        return buf, re.astype(np.float64) + 1j * im.astype(np.float64)
+
+    A, Ac = operand(M, transA, 1e30)
+    B, Bc = operand(N, transB, -1e30)
+    ldc = r4(N)
     Ad, Bd = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
     Cd = torch.full((bins, 2, M, ldc), float("nan"), device="cuda")
     status = torch.zeros(64, dtype=torch.int32, device="cuda")
-    fc.fftconv_bin_contract(Ad, Bd, Cd, K, math=math, status_word=status)
+    fc.fftconv_bin_contract(Ad, Bd, Cd, M, N, K, transA, transB, conjA, conjB, math=math,
+                            status_word=status)
     torch.cuda.synchronize()
     assert int(status[0].item()) == 0
     C = Cd.cpu().numpy().astype(np.float64)
     got = C[:, 0, :, :N] + 1j * C[:, 1, :, :N]
-    Ac = A[:, 0, :, :K].astype(np.float64) + 1j * A[:, 1, :, :K].astype(np.float64)
-    Bc = B[:, 0, :, :K].astype(np.float64) + 1j * B[:, 1, :, :K].astype(np.float64)
-    ref = oracle.bin_contract(Ac, Bc, False, False)
+    ref = oracle.bin_contract(Ac, Bc, conjA, conjB)
     assert np.all(np.isfinite(got.real)) and np.all(np.isfinite(got.imag))
-    # columns beyond N in the padded leading dimension stay untouched
+    # padding columns of C (N..ldc-1) are scratch: untouched or zero, never data
     if ldc > N:
-        assert np.all(np.isnan(C[..., N:]))
+        pad = C[..., N:]
+        assert np.all(np.isnan(pad) | (pad == 0))
     return float(np.max(np.abs(got - ref)) / np.max(np.abs(ref)))
 
 
@@ -61,3 +70,20 @@ def test_contraction_tf32_tensor_cores(shape):
 def test_tf32_many_tiles_per_cta():
     # more tiles than SMs: every CTA walks several tiles through both accumulator buffers
     assert run(700, 128, 128, 64, math=2, seed=3) <= TOL[2]
+
+
+# operand storage / conjugation as used by the three passes, plus the remaining combinations
+FLAGS = [
+    dict(transA=False, transB=False, conjA=False, conjB=True),    # fprop
+    dict(transA=False, transB=True, conjA=False, conjB=False),    # bprop
+    dict(transA=True, transB=True, conjA=True, conjB=False),      # accGrad
+    dict(transA=True, transB=False, conjA=True, conjB=True),
+]
+
+
+@pytest.mark.parametrize("flags", FLAGS)
+@pytest.mark.parametrize("math", [1, 2])
+@pytest.mark.parametrize("shape", [(5, 128, 128, 64), (3, 130, 70, 33), (2, 37, 129, 100),
+                                   (4, 64, 96, 128), (2, 8, 8, 4)])
+def test_contraction_layouts_and_conjugates(shape, math, flags):
+    assert run(*shape, math=math, seed=9, **flags) <= TOL[math]
