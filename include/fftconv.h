@@ -140,11 +140,12 @@ int fft2d_c2r(const void* in_c, float* out, int batch, int n, int oh, int ow, fl
  *   C[b][m][nn] = sum_k op(A)[b][m][k] * op(B)[b][nn][k]
  * with op = identity, or the complex conjugate when conjA / conjB is non-zero
  * (Section 2: the conjugate turns the product into a cross-correlation).
- * Operands are planar device arrays, plane 0 real and plane 1 imaginary:
- *   A: [bins][2][M][lda], k contiguous (lda >= K); with transA != 0 it is stored
- *      [bins][2][K][lda], m contiguous (lda >= M);
- *   B: [bins][2][N][ldb] (ldb >= K), or with transB != 0 [bins][2][K][ldb] (ldb >= N);
- *   C: [bins][2][M][ldc], ldc >= N; the padding columns N..ldc-1 are scratch
+ * Operands are planar device arrays: the real matrices of all bins first, then
+ * the imaginary matrices of all bins:
+ *   A: [2][bins][M][lda], k contiguous (lda >= K); with transA != 0 it is stored
+ *      [2][bins][K][lda], m contiguous (lda >= M);
+ *   B: [2][bins][N][ldb] (ldb >= K), or with transB != 0 [2][bins][K][ldb] (ldb >= N);
+ *   C: [2][bins][M][ldc], ldc >= N; the padding columns N..ldc-1 are scratch
  *      (they may be overwritten with zeros).
  * lda, ldb, ldc must be multiples of 4 and the pointers 16-byte aligned.
  * math: FFTCONV_MATH_FP32 or FFTCONV_MATH_TF32 (AUTO resolves by shape).

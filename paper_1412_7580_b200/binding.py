@@ -224,10 +224,10 @@ def fft2d_c2r(in_c, out, n, scale, accumulate=False, stream=None) -> None:
 
 def fftconv_bin_contract(A, B, C, M, N, K, transA=False, transB=False, conjA=False, conjB=False,
                          math=MATH_FP32, status_word=None, stream=None) -> None:
-    """Planar float32 operands: A [bins, 2, M, lda] (or [bins, 2, K, lda] with transA),
-    B [bins, 2, N, ldb] (or [bins, 2, K, ldb] with transB), C [bins, 2, M, ldc]."""
-    bins = A.shape[0]
-    assert A.shape[1] == 2 and B.shape[:2] == (bins, 2) and C.shape[:3] == (bins, 2, M)
+    """Planar float32 operands: A [2, bins, M, lda] (or [2, bins, K, lda] with transA),
+    B [2, bins, N, ldb] (or [2, bins, K, ldb] with transB), C [2, bins, M, ldc]."""
+    bins = A.shape[1]
+    assert A.shape[0] == 2 and B.shape[:2] == (2, bins) and C.shape[:3] == (2, bins, M)
     assert A.shape[2] == (K if transA else M) and B.shape[2] == (K if transB else N)
     lda, ldb, ldc = A.shape[3], B.shape[3], C.shape[3]
     sw = ctypes.c_void_p(status_word.data_ptr()) if status_word is not None else ctypes.c_void_p()

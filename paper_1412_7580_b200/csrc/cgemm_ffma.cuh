@@ -2,9 +2,10 @@
 //
 // For every bin b:  C[b][m][n] = sum_k op(A)[b][m][k] * op(B)[b][n][k]  (complex;
 // op = identity or complex conjugate).
-// Operands are planar (plane 0 real, plane 1 imaginary).  A is [bins][2][M][lda]
-// (k contiguous) or, with transA, [bins][2][K][lda] (m contiguous); B likewise
-// [bins][2][N][ldb] or, with transB, [bins][2][K][ldb]; C is [bins][2][M][ldc].
+// Operands are planar: all real matrices of the bins first, then all imaginary
+// ones.  A is [2][bins][M][lda] (k contiguous) or, with transA, [2][bins][K][lda]
+// (m contiguous); B likewise [2][bins][N][ldb] or, with transB, [2][bins][K][ldb];
+// C is [2][bins][M][ldc].
 //
 // CTA tile 64 x 64 of one bin, 256 threads, each thread a 4 x 4 block of complex
 // outputs (64 FFMAs per k against four 16-byte shared loads).  This is the exact
@@ -37,9 +38,11 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
     const size_t planeA = (size_t)(p.transA ? p.K : p.M) * p.lda,
                  planeB = (size_t)(p.transB ? p.K : p.N) * p.ldb, planeC = (size_t)p.M * p.ldc;
     const float sa = p.conjA ? -1.0f : 1.0f, sb = p.conjB ? -1.0f : 1.0f;
-    const float* Ab = p.A + (size_t)bin * 2 * planeA;
-    const float* Bb = p.B + (size_t)bin * 2 * planeB;
-    float* Cb = p.C + (size_t)bin * 2 * planeC;
+    const float* Ab = p.A + (size_t)bin * planeA;
+    const float* Bb = p.B + (size_t)bin * planeB;
+    float* Cb = p.C + (size_t)bin * planeC;
+    const size_t imA = (size_t)p.bins * planeA, imB = (size_t)p.bins * planeB,
+                 imC = (size_t)p.bins * planeC;
 
     const int tx = tid & 15, ty = tid >> 4;      // 16 x 16 threads
     const int lk = tid & 15, lr = tid >> 4;      // loader: k within chunk, row group
@@ -61,7 +64,7 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
                 float are = 0.f, aim = 0.f;
                 if (k < p.K && m < p.M) {
                     are = __ldg(Ab + (size_t)m * p.lda + k);
-                    aim = sa * __ldg(Ab + planeA + (size_t)m * p.lda + k);
+                    aim = sa * __ldg(Ab + imA + (size_t)m * p.lda + k);
                 }
                 sA[0][lk][r] = are; sA[1][lk][r] = aim;
             }
@@ -73,7 +76,7 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
                 float are = 0.f, aim = 0.f;
                 if (k < p.K && m < p.M) {
                     are = __ldg(Ab + (size_t)k * p.lda + m);
-                    aim = sa * __ldg(Ab + planeA + (size_t)k * p.lda + m);
+                    aim = sa * __ldg(Ab + imA + (size_t)k * p.lda + m);
                 }
                 sA[0][kk][r] = are; sA[1][kk][r] = aim;
             }
@@ -86,7 +89,7 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
                 float bre = 0.f, bim = 0.f;
                 if (k < p.K && n < p.N) {
                     bre = __ldg(Bb + (size_t)n * p.ldb + k);
-                    bim = sb * __ldg(Bb + planeB + (size_t)n * p.ldb + k);
+                    bim = sb * __ldg(Bb + imB + (size_t)n * p.ldb + k);
                 }
                 sB[0][lk][r] = bre; sB[1][lk][r] = bim;
             }
@@ -98,7 +101,7 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
                 float bre = 0.f, bim = 0.f;
                 if (k < p.K && n < p.N) {
                     bre = __ldg(Bb + (size_t)k * p.ldb + n);
-                    bim = sb * __ldg(Bb + planeB + (size_t)k * p.ldb + n);
+                    bim = sb * __ldg(Bb + imB + (size_t)k * p.ldb + n);
                 }
                 sB[0][kk][r] = bre; sB[1][kk][r] = bim;
             }
@@ -133,7 +136,7 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
         const int m = m_blk + ty * 4 + i;
         if (m >= p.M) continue;
         float* o_r = Cb + (size_t)m * p.ldc + n0;
-        float* o_i = o_r + planeC;
+        float* o_i = o_r + imC;
         if (n0 + 3 < p.N) {
             *reinterpret_cast<float4*>(o_r) = make_float4(cr[i][0], cr[i][1], cr[i][2], cr[i][3]);
             *reinterpret_cast<float4*>(o_i) = make_float4(ci[i][0], ci[i][1], ci[i][2], ci[i][3]);

@@ -35,6 +35,7 @@
 #include <stdint.h>
 
 #include "cgemm_ffma.cuh"
+#include "tma_util.cuh"
 
 namespace fc {
 
@@ -236,21 +237,21 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                     for (int part = 0; part < 2; ++part) {
                         if constexpr (!TA) {
                             tma_load_3d(dst + part * TC_TILE_BYTES, &tmA, kb * TC_BK, m_t * TC_BM,
-                                        2 * bin + part, full(s));
+                                        part * p.bins + bin, full(s));
                         } else {
 #pragma unroll
                             for (int blk = 0; blk < 4; ++blk)
                                 tma_load_3d(dst + part * TC_TILE_BYTES + blk * 4096, &tmA,
-                                            m_t * TC_BM + blk * 32, kb * TC_BK, 2 * bin + part, full(s));
+                                            m_t * TC_BM + blk * 32, kb * TC_BK, part * p.bins + bin, full(s));
                         }
                         if constexpr (!TB) {
                             tma_load_3d(dst + (2 + part) * TC_TILE_BYTES, &tmB, kb * TC_BK, n_t * TC_BN,
-                                        2 * bin + part, full(s));
+                                        part * p.bins + bin, full(s));
                         } else {
 #pragma unroll
                             for (int blk = 0; blk < 4; ++blk)
                                 tma_load_3d(dst + (2 + part) * TC_TILE_BYTES + blk * 4096, &tmB,
-                                            n_t * TC_BN + blk * 32, kb * TC_BK, 2 * bin + part, full(s));
+                                            n_t * TC_BN + blk * 32, kb * TC_BK, part * p.bins + bin, full(s));
                         }
                     }
                 }
@@ -359,7 +360,7 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                         __syncwarp();
                         if (lane == 0) {
-                            tma_store_3d(&tmC, sbuf, col0 + c, row0, 2 * bin + part);
+                            tma_store_3d(&tmC, sbuf, col0 + c, row0, part * p.bins + bin);
                             asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                         }
                         ++nstore;
@@ -384,42 +385,6 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 }
 
 // ---- host side -------------------------------------------------------------
-typedef CUresult (*tc_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                 const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                 const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static tc_encode_fn tc_get_encode() {
-    static tc_encode_fn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) ==
-                cudaSuccess && qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<tc_encode_fn>(sym);
-    }
-    return fn;
-}
-
-// Planar matrix family [bins][2][rows][ld] seen as a 3-D tensor (col, row,
-// bin*2+part) with `cols` valid columns; out-of-range coordinates read as zero
-// and are clipped on store, which is what makes ragged M, N, K work.
-static bool tc_make_map(CUtensorMap* map, const float* base, int bins, int rows, int cols, int ld,
-                        int box_cols, int box_rows,
-                        CUtensorMapSwizzle swz = CU_TENSOR_MAP_SWIZZLE_128B) {
-    tc_encode_fn enc = tc_get_encode();
-    if (!enc) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)bins * 2};
-    cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)rows * ld * 4};
-    cuuint32_t box[3] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides,
-               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
-               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <bool TA, bool TB>
 static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStream_t st, int sm_count) {
     auto kern = cgemm_tc_kernel<TA, TB>;

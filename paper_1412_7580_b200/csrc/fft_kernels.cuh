@@ -1,34 +1,56 @@
 // Batched 2-D R2C / C2R FFT kernels with fused zero-padding, fused
 // frequency-major transpose, crop, scale and accumulate.
 //
-// One CTA transforms a tile of G planes that are adjacent along the *minor*
-// index of the frequency-major matrix they are written to (read from), so that
-// every frequency bin receives G consecutive floats: the transposition
-// BDHW -> HWBD of the paper's Table 1 happens in the store (load) itself and no
-// separate transpose pass or padded tensor exists (Section 5.1: zero-copy
-// padding by clipped loads; Section 5.1: transposed output removes a pass).
+// One CTA transforms tiles of G planes that are adjacent along the minor index
+// of the frequency-major matrix they are written to (read from), so that every
+// frequency bin receives G consecutive floats: the transposition BDHW -> HWBD of
+// the paper's Table 1 happens in the store (load) itself and no separate
+// transpose pass or padded tensor exists (Section 5.1: zero-copy padding by
+// clipped loads; returning the transposed spectrum removes a pass).
 //
-// Structure of the forward kernel (the inverse mirrors it):
-//   1. coalesced copy of the G real planes into shared memory;
-//   2. one thread per non-zero row: real FFT of length N in registers
-//      (a complex FFT of length N/2 plus a Hermitian post-pass), half spectrum
-//      (N/2+1 bins) written back to shared memory;
-//   3. N/2 column transforms per plane -- columns 0 and N/2 are real and ride
-//      together as one complex column (the paper's "n x n/2 with border case",
-//      Section 5.2) -- each split over two threads by one
-//      decimation-in-frequency step applied while loading, then an N/2-point
-//      register FFT; results go straight from registers to global memory,
-//      lanes running over the G planes.
+// Frequency bins.  For a real plane only half the spectrum is kept (Section 3.1).
+// Inside the convolution passes the kept half is ky in [0, n/2], kx in [0, n),
+// numbered bin = kx*(n/2+1) + ky, because the first 1-D pass then runs down the
+// columns of the plane with one thread per column, which reads shared memory
+// without bank conflicts for every plane width and lets the planes be staged by
+// one bulk asynchronous copy.  The per-bin contraction does not care which half
+// is kept or how bins are numbered.  The bare transforms present the
+// conventional [n][n/2+1] half instead; the kernels translate through the
+// Hermitian symmetry X[ky][kx] = conj X[-ky][-kx].
+//
+// Spectra in global memory are planar: [2][bins][R][ld] floats, all real parts
+// first.  A tile's spectrum is assembled in shared memory as [part][bin][G] and
+// moved by the TMA as boxes of G columns x 1 row x D bins, so the SM never
+// issues a scattered global access and every shared-memory access of a warp is
+// one contiguous 128-byte line with an immediate offset.
+//
+// Forward kernel, per tile (the inverse mirrors it):
+//   1. bulk asynchronous copy of the G real planes into shared memory; the copy
+//      of the next tile is issued as soon as step 2 has read the current one;
+//   2. one thread per non-zero column: real FFT of length N down the column, in
+//      registers (complex FFT of length N/2 plus a Hermitian post-pass), half
+//      spectrum (N/2+1 rows) written back to shared memory;
+//   3. N/2 row transforms per plane -- rows ky = 0 and ky = N/2 are real and ride
+//      together as one complex row (the paper's "n x n/2 with border case",
+//      Section 5.2) -- each split over two threads by one decimation-in-frequency
+//      step applied while loading, then an N/2-point register FFT; results go to
+//      the staging tile and from there to global memory by TMA stores.
+// CTAs are persistent and walk the tiles with a grid stride.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "fft_core.cuh"
+#include "tma_util.cuh"
 
 namespace fc {
 
-enum { LAYOUT_FREQ_MAJOR = 0, LAYOUT_BARE = 1 };
+// LAYOUT_FREQ_TMA / _DIRECT: planar frequency-major spectra, moved by the TMA or
+// by plain per-thread accesses; LAYOUT_BARE: [plane][n][n/2+1] interleaved pairs.
+enum { LAYOUT_FREQ_TMA = 0, LAYOUT_BARE = 1, LAYOUT_FREQ_DIRECT = 2 };
 
 struct FftParams {
     const float* real_in;   // forward: real planes in
@@ -36,451 +58,590 @@ struct FftParams {
     const float* spec_in;   // inverse: spectra in
     float* spec_out;        // forward: spectra out
     int h, w;               // forward: plane size; inverse: crop window (hc, wc)
-    int R, C;               // frequency-major matrix: rows, cols (planes = R*C)
+    int R, C;               // frequency-major matrix: rows, cols (plane = row*C + col)
     int ld;                 // its leading dimension in floats
-    long long in_rs, in_cs; // forward: input plane index = row*in_rs + col*in_cs
-    int conj;               // forward: negate imaginary parts on store
     int tiles_per_row;      // ceil(C / G)
-    int pitch;              // shared-memory plane pitch in complex elements
+    int num_tiles;          // R * tiles_per_row
+    int in_bytes;           // shared-memory bytes reserved for the real tile (multiple of 128)
     float scale;            // inverse
     int accumulate;         // inverse
 };
 
-// Shared-memory pitch of one plane's half spectrum (rows x (N/2+1) complex)
-// such that lanes running over g (and then over adjacent columns) hit distinct
-// 8-byte banks: pitch = (16 / min(G,16)) * odd.
-static inline int smem_plane_pitch(int rows, int N, int G) {
-    int need = rows * (N / 2 + 1);
-    int unit = 16 / (G < 16 ? G : 16);
-    int m = (need + unit - 1) / unit;
-    if ((m & 1) == 0) ++m;
-    return m * unit;
+// Geometry of the half-spectrum scratch ("mid") of one plane in shared memory:
+// (N/2+1) rows of N+1 complex, plane pitch = (16 / min(G,16)) * odd so that lanes
+// running over the plane index and then over adjacent rows hit distinct 8-byte
+// banks.
+template <int N, int G>
+struct MidGeom {
+    static constexpr int PW = N + 1;
+    static constexpr int NEED = (N / 2 + 1) * PW;
+    static constexpr int UNIT = 16 / (G < 16 ? G : 16);
+    static constexpr int MUL = ((NEED + UNIT - 1) / UNIT) | 1;
+    static constexpr int P = MUL * UNIT;
+    static constexpr int BYTES = ((G * P * 8 + 127) / 128) * 128;
+};
+// Bins moved per TMA box: the largest divisor of N*(N/2+1) that is <= 256.
+constexpr int tma_bins_per_box(int N) {
+    int B = N * (N / 2 + 1), best = 1;
+    for (int d = 1; d <= 256; ++d)
+        if (B % d == 0) best = d;
+    return best;
+}
+static inline int real_tile_bytes(int G, int rows, int cols) {
+    return (G * rows * cols * 4 + 127) & ~127;
 }
 
-static inline size_t r2c_smem_bytes(int N, int G, int h, int w) {
-    size_t a = (size_t)G * h * (w | 1) * sizeof(float);
-    size_t b = (size_t)G * smem_plane_pitch(h, N, G) * sizeof(float2);
-    return a > b ? a : b;
+// ---- small PTX helpers (bulk asynchronous copies) ---------------------------
+__device__ __forceinline__ uint32_t fk_smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
-static inline size_t c2r_smem_bytes(int N, int G, int hc, int wc) {
-    return r2c_smem_bytes(N, G, hc, wc);
+__device__ __forceinline__ void fk_mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fk_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool fk_mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait (about a second); returns false when it ran out.
+__device__ __forceinline__ bool fk_mbar_wait(uint32_t bar, uint32_t parity) {
+    if (fk_mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+        for (int i = 0; i < 64; ++i)
+            if (fk_mbar_try_wait(bar, parity)) return true;
+        if (clock64() - t0 > 2000000000LL) return false;
+    }
+}
+__device__ __forceinline__ void fk_bulk_g2s(uint32_t dst, const void* src, uint32_t bytes,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fk_tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                               int c2, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void fk_tma_store_3d(const CUtensorMap* map, uint32_t src, int c0,
+                                                int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+__device__ __forceinline__ void fk_bulk_commit() {
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void fk_bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
 
-// Copy `count` planes of rows x cols floats between a contiguous global range
-// (plane stride rows*cols) and shared memory with row pitch colsp.
-// TO_SMEM: global -> shared; otherwise shared -> global (optionally adding).
-template <int T, bool TO_SMEM>
-__device__ __forceinline__ void copy_planes(float* smem, const float* gsrc, float* gdst,
-                                            int count, long long plane_stride, int rows,
-                                            int cols, int colsp, float scale, int accumulate) {
-    const int hw = rows * cols;
-    const int tid = threadIdx.x;
-    if (colsp == cols && plane_stride == hw) {
-        const int total = count * hw;
-        const uintptr_t addr = TO_SMEM ? (uintptr_t)gsrc : (uintptr_t)gdst;
-        if ((addr & 15) == 0) {
-            const int total4 = total >> 2;
-            if constexpr (TO_SMEM) {
-                const float4* s4 = reinterpret_cast<const float4*>(gsrc);
-                float4* d4 = reinterpret_cast<float4*>(smem);
-                for (int i = tid; i < total4; i += T) d4[i] = __ldg(s4 + i);
-                for (int i = (total4 << 2) + tid; i < total; i += T) smem[i] = __ldg(gsrc + i);
+// One decimation-in-frequency step fused into the loads of an N-point complex
+// transform split over two threads (q = 0: even outputs, q = 1: odd outputs).
+template <int N, bool INV, int Q, class Load>
+__device__ __forceinline__ void load_split(Load&& load, float (&ar)[N / 2], float (&ai)[N / 2]) {
+    constexpr int M = N / 2;
+    static_for<M>([&](auto J) {
+        constexpr int j = decltype(J)::value;
+        const float2 lo = load(J), hi = load(std::integral_constant<int, j + M>{});
+        if constexpr (Q == 0) {
+            ar[j] = lo.x + hi.x;
+            ai[j] = lo.y + hi.y;
+        } else {
+            const float dr = lo.x - hi.x, di = lo.y - hi.y;
+            if constexpr (j == 0) {
+                ar[j] = dr; ai[j] = di;
+            } else if constexpr (4 * j == N) {
+                if constexpr (!INV) { ar[j] = di; ai[j] = -dr; }
+                else                { ar[j] = -di; ai[j] = dr; }
             } else {
-                const float4* s4 = reinterpret_cast<const float4*>(smem);
-                float4* d4 = reinterpret_cast<float4*>(gdst);
-                for (int i = tid; i < total4; i += T) {
-                    float4 v = s4[i];
-                    v.x *= scale; v.y *= scale; v.z *= scale; v.w *= scale;
-                    if (accumulate) {
-                        float4 o = d4[i];
-                        v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
-                    }
-                    d4[i] = v;
-                }
-                for (int i = (total4 << 2) + tid; i < total; i += T) {
-                    float v = smem[i] * scale;
-                    if (accumulate) v += gdst[i];
-                    gdst[i] = v;
-                }
-            }
-        } else {
-            for (int i = tid; i < total; i += T) {
-                if constexpr (TO_SMEM) {
-                    smem[i] = __ldg(gsrc + i);
-                } else {
-                    float v = smem[i] * scale;
-                    if (accumulate) v += gdst[i];
-                    gdst[i] = v;
-                }
+                constexpr float c = Tw<N, j>::c;
+                constexpr float s = INV ? -Tw<N, j>::s : Tw<N, j>::s;
+                ar[j] = fc_fma(s, di, c * dr);
+                ai[j] = fc_fma(-s, dr, c * di);
             }
         }
-        return;
-    }
-    // general case: walk (g, r, c) incrementally, T elements per step
-    int g = tid / hw;
-    int rem = tid - g * hw;
-    int r = rem / cols;
-    int c = rem - r * cols;
-    const int dg = T / hw;
-    const int drem = T - dg * hw;
-    const int dr = drem / cols;
-    const int dc = drem - dr * cols;
-    while (g < count) {
-        const long long gi = (long long)g * plane_stride + r * cols + c;
-        const int si = (g * rows + r) * colsp + c;
-        if constexpr (TO_SMEM) {
-            smem[si] = __ldg(gsrc + gi);
-        } else {
-            float v = smem[si] * scale;
-            if (accumulate) v += gdst[gi];
-            gdst[gi] = v;
-        }
-        c += dc; r += dr;
-        if (c >= cols) { c -= cols; ++r; }
-        g += dg;
-        if (r >= rows) { r -= rows; ++g; }
-    }
+    });
 }
 
 // ---------------------------------------------------------------------------
 // Forward: real planes -> half spectra.
+// ALIAS: the half-spectrum scratch overwrites the staging area of the real tile
+// (no prefetch of the next tile); used where one tile nearly fills shared memory.
 // ---------------------------------------------------------------------------
-template <int N, int G, int LAYOUT>
-__global__ void __launch_bounds__(N* G) r2c_kernel(const FftParams p) {
-    constexpr int T = N * G, NC = N / 2 + 1, M = N / 2, HALF = T / 2;
-    static_assert(HALF % 32 == 0, "the two halves of a column transform must be warp-uniform");
-    extern __shared__ __align__(16) unsigned char fc_smem[];
+template <int N, int G, int LAYOUT, bool ALIAS, int MINB>
+__global__ void __launch_bounds__(N* G, MINB)
+r2c_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
+    constexpr int T = N * G, NC = N / 2 + 1, M = N / 2, HALF = T / 2, B = N * NC;
+    constexpr int PW = MidGeom<N, G>::PW, P = MidGeom<N, G>::P;
+    constexpr bool TMA = (LAYOUT == LAYOUT_FREQ_TMA);
+    constexpr int D = tma_bins_per_box(N);
+    static_assert(HALF % 32 == 0, "the two halves of a row transform must be warp-uniform");
+    extern __shared__ __align__(128) unsigned char fc_smem[];
     float* sIn = reinterpret_cast<float*>(fc_smem);
-    float2* sMid = reinterpret_cast<float2*>(fc_smem);
+    unsigned char* mid_base = fc_smem + (ALIAS ? 0 : p.in_bytes);
+    float2* sMid = reinterpret_cast<float2*>(mid_base);
+    float* sStage = reinterpret_cast<float*>(
+        mid_base + (ALIAS ? (p.in_bytes > MidGeom<N, G>::BYTES ? p.in_bytes : MidGeom<N, G>::BYTES)
+                          : MidGeom<N, G>::BYTES));
+    __shared__ __align__(8) unsigned long long bar_storage;
+    const uint32_t bar = fk_smem_u32(&bar_storage);
 
     const int tid = threadIdx.x;
-    const int row = blockIdx.x / p.tiles_per_row;
-    const int c0 = (blockIdx.x - row * p.tiles_per_row) * G;
-    const int gcount = min(G, p.C - c0);
-    const int h = p.h, w = p.w, wp = w | 1, P = p.pitch;
+    const int h = p.h, w = p.w, hw = h * w;
+    // thread roles, fixed for the whole kernel
+    const int gA = tid / w, cA = tid - gA * w;                  // step 2: (plane, column)
+    const int q = tid / HALF, u = tid - q * HALF;               // step 3: (half, row ky, plane)
+    const int kyp = u / G, gB = u - kyp * G;
 
-    // 1. stage the tile's planes (only the h x w non-zero part exists anywhere)
-    {
-        const long long first = (long long)row * p.in_rs + (long long)c0 * p.in_cs;
-        copy_planes<T, true>(sIn, p.real_in + first * h * w, nullptr, gcount,
-                             p.in_cs * h * w, h, w, wp, 1.0f, 0);
+    if (tid == 0) {
+        fk_mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (!ALIAS) {
+        // columns >= w of the scratch are never written: zero them once, read them freely
+        for (int i = tid; i < G * P; i += T) sMid[i] = make_float2(0.0f, 0.0f);
     }
     __syncthreads();
 
-    // 2. row transforms: thread = (plane g, row r), r < h
-    {
-        const int g = tid / h, r = tid - g * h;
-        const bool act = (tid < G * h) && (g < gcount);
-        float Xr[NC], Xi[NC];
-        if (act) {
-            float v[N];
-            const float* src = sIn + (g * h + r) * wp;
-            static_for<N>([&](auto Cc) {
+    // Stage the planes of `tile`.  Returns true if the copy is asynchronous (wait on the
+    // barrier before reading), false if it was done with plain loads by all threads.
+    auto stage = [&](int tile) -> bool {
+        const int row = tile / p.tiles_per_row;
+        const int c0 = (tile - row * p.tiles_per_row) * G;
+        const int gcount = min(G, p.C - c0);
+        const float* src = p.real_in + ((size_t)row * p.C + c0) * hw;
+        const int total = gcount * hw;
+        if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+            const int bulk = total & ~3;
+            if (tid == 0 && bulk > 0) {
+                fk_mbar_expect_tx(bar, (uint32_t)bulk * 4u);
+                fk_bulk_g2s(fk_smem_u32(sIn), src, (uint32_t)bulk * 4u, bar);
+            }
+            if (tid < total - bulk) sIn[bulk + tid] = __ldg(src + bulk + tid);
+            return bulk > 0;
+        }
+        for (int i = tid; i < total; i += T) sIn[i] = __ldg(src + i);
+        return false;
+    };
+
+    uint32_t phase = 0;
+    bool pending = false, store_pending = false;
+    if (blockIdx.x < p.num_tiles) pending = stage(blockIdx.x);
+    __syncthreads();           // plain-load parts of the first tile are visible to everyone
+
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+        const int row = tile / p.tiles_per_row;
+        const int c0 = (tile - row * p.tiles_per_row) * G;
+        const int gcount = min(G, p.C - c0);
+
+        if (pending) {
+            if (!fk_mbar_wait(bar, phase)) return;     // copy never landed: give up
+            phase ^= 1u;
+        }
+
+        // 2. column transforms: thread = (plane gA, column cA), cA < w
+        {
+            const bool act = (gA < gcount);             // gA < G follows from tid < G*w
+            float Xr[NC], Xi[NC];
+            if (act) {
+                float v[N];
+                const float* src = sIn + gA * hw + cA;
+                static_for<N>([&](auto Rr) {
+                    constexpr int r = decltype(Rr)::value;
+                    v[r] = (r < h) ? src[r * w] : 0.0f;
+                });
+                rfft<N>(v, Xr, Xi);
+            }
+            if (TMA && store_pending && tid == 0) fk_bulk_wait_read();   // staging tile free again
+            __syncthreads();   // tile consumed (and the previous tile's step 3 is done with sMid)
+            const int next = tile + gridDim.x;
+            if (!ALIAS) pending = (next < p.num_tiles) ? stage(next) : false;
+            if (act) {
+                float2* dst = sMid + gA * P + cA;
+                static_for<NC>([&](auto Kk) {
+                    constexpr int k = decltype(Kk)::value;
+                    dst[k * PW] = make_float2(Xr[k], Xi[k]);
+                });
+            }
+        }
+        __syncthreads();
+
+        // 3. row transforms: thread = (half q, row kyp, plane gB)
+        if (TMA || gB < gcount) {
+            float ar[M], ai[M];
+            const float2* rowp = sMid + gB * P + kyp * PW;
+            const bool packed = (kyp == 0);
+            auto load = [&](auto Cc) -> float2 {
                 constexpr int c = decltype(Cc)::value;
-                v[c] = (c < w) ? src[c] : 0.0f;
-            });
-            rfft<N>(v, Xr, Xi);
-        }
-        __syncthreads();   // every row is in registers: the staging area may be overwritten
-        if (act) {
-            float2* dst = sMid + g * P + r * NC;
-            static_for<NC>([&](auto Kk) {
-                constexpr int k = decltype(Kk)::value;
-                dst[k] = make_float2(Xr[k], Xi[k]);
-            });
-        }
-    }
-    __syncthreads();
-
-    // 3. column transforms: thread = (half q, column kxp, plane g)
-    const int q = tid / HALF;
-    const int u = tid - q * HALF;
-    const int kxp = u / G;
-    const int g = u - kxp * G;
-    if (g >= gcount) return;
-
-    float ar[M], ai[M];
-    {
-        const float2* col = sMid + g * P + kxp;
-        const bool packed = (kxp == 0);
-        auto load = [&](int r) -> float2 {
-            if (r >= h) return make_float2(0.0f, 0.0f);
-            float2 v = col[r * NC];
-            if (packed) v.y = col[r * NC + M].x;   // Nyquist column rides as the imaginary part
-            return v;
-        };
-        auto split = [&](auto Q) {
-            constexpr int qq = decltype(Q)::value;
-            static_for<M>([&](auto J) {
-                constexpr int j = decltype(J)::value;
-                const float2 lo = load(j), hi = load(j + M);
-                if constexpr (qq == 0) {
-                    ar[j] = lo.x + hi.x;
-                    ai[j] = lo.y + hi.y;
-                } else {
-                    const float dr = lo.x - hi.x, di = lo.y - hi.y;
-                    if constexpr (j == 0) {
-                        ar[j] = dr; ai[j] = di;
-                    } else if constexpr (4 * j == N) {
-                        ar[j] = di; ai[j] = -dr;
-                    } else {
-                        constexpr float c = Tw<N, j>::c;
-                        constexpr float s = Tw<N, j>::s;
-                        ar[j] = fc_fma(s, di, c * dr);
-                        ai[j] = fc_fma(-s, dr, c * di);
-                    }
+                float2 v;
+                if constexpr (ALIAS) {
+                    if (c >= w) return make_float2(0.0f, 0.0f);
                 }
-            });
-        };
-        if (q == 0) split(std::integral_constant<int, 0>{});
-        else        split(std::integral_constant<int, 1>{});
-    }
-    cfft<M, false>(ar, ai);   // ar/ai[k] = F[2k+q]
+                v = rowp[c];
+                if (packed) v.y = rowp[M * PW + c].x;   // row ky = N/2 rides as the imaginary part
+                return v;
+            };
+            if (q == 0) load_split<N, false, 0>(load, ar, ai);
+            else        load_split<N, false, 1>(load, ar, ai);
+            cfft<M, false>(ar, ai);                     // ar/ai[k] = F[kx = 2k+q]
 
-    const float sgn = p.conj ? -1.0f : 1.0f;
-    if constexpr (LAYOUT == LAYOUT_FREQ_MAJOR) {
-        const size_t plane = (size_t)p.R * p.ld;               // one re or im matrix
-        float* base = p.spec_out + (size_t)row * p.ld + c0 + g;
-        if (kxp != 0) {
-            static_for<M>([&](auto Kk) {
-                constexpr int k = decltype(Kk)::value;
-                const int ky = 2 * k + q;
-                float* o = base + (size_t)(ky * NC + kxp) * 2 * plane;
-                o[0] = ar[k];
-                o[plane] = sgn * ai[k];
-            });
-        } else {
-            auto untangle = [&](auto Q) {
-                constexpr int qq = decltype(Q)::value;
-                static_for<M>([&](auto Kk) {
-                    constexpr int k = decltype(Kk)::value;
-                    constexpr int kp = (qq == 0) ? ((M - k) % M) : (M - 1 - k);
-                    constexpr int ky = 2 * k + qq;
-                    const float fr = ar[k], fi = ai[k], gr = ar[kp], gi = ai[kp];
-                    float* o0 = base + (size_t)(ky * NC) * 2 * plane;
-                    float* oN = base + (size_t)(ky * NC + M) * 2 * plane;
-                    o0[0] = 0.5f * (fr + gr);
-                    o0[plane] = sgn * 0.5f * (fi - gi);
-                    oN[0] = 0.5f * (fi + gi);
-                    oN[plane] = sgn * 0.5f * (gr - fr);
-                });
-            };
-            if (q == 0) untangle(std::integral_constant<int, 0>{});
-            else        untangle(std::integral_constant<int, 1>{});
+            if constexpr (LAYOUT != LAYOUT_BARE) {
+                // element (part, bin = kx*NC + ky, plane g): staging offset (part*B + bin)*G + g,
+                // global offset ((part*B + bin)*R + row)*ld + col
+                float* o;
+                size_t sb, sp;      // strides of one bin and of one part
+                if constexpr (TMA) {
+                    o = sStage + (q * NC + kyp) * G + gB;
+                    sb = G; sp = (size_t)B * G;
+                } else {
+                    const size_t mat = (size_t)p.R * p.ld;
+                    o = p.spec_out + (size_t)(q * NC + kyp) * mat + (size_t)row * p.ld + c0 + gB;
+                    sb = mat; sp = (size_t)B * mat;
+                }
+                if (!packed) {
+                    static_for<M>([&](auto Kk) {
+                        constexpr int k = decltype(Kk)::value;
+                        o[(size_t)(2 * k * NC) * sb] = ar[k];
+                        o[(size_t)(2 * k * NC) * sb + sp] = ai[k];
+                    });
+                } else {
+                    auto untangle = [&](auto Q) {
+                        constexpr int qq = decltype(Q)::value;
+                        static_for<M>([&](auto Kk) {
+                            constexpr int k = decltype(Kk)::value;
+                            constexpr int kp = (qq == 0) ? ((M - k) % M) : (M - 1 - k);
+                            const float fr = ar[k], fi = ai[k], gr = ar[kp], gi = ai[kp];
+                            float* o0 = o + (size_t)(2 * k * NC) * sb;      // row ky = 0
+                            float* oN = o0 + (size_t)M * sb;                // row ky = N/2
+                            o0[0] = 0.5f * (fr + gr);
+                            o0[sp] = 0.5f * (fi - gi);
+                            oN[0] = 0.5f * (fi + gi);
+                            oN[sp] = 0.5f * (gr - fr);
+                        });
+                    };
+                    if (q == 0) untangle(std::integral_constant<int, 0>{});
+                    else        untangle(std::integral_constant<int, 1>{});
+                }
+            } else {
+                // conventional half [ky][kx <= N/2]; the other rows come from the mirror bin
+                float2* base = reinterpret_cast<float2*>(p.spec_out) +
+                               ((size_t)row * p.C + c0 + gB) * (size_t)(N * NC);
+                if (!packed) {
+                    static_for<M>([&](auto Kk) {
+                        constexpr int k = decltype(Kk)::value;
+                        const int kx = 2 * k + q;
+                        if (kx <= M) base[kyp * NC + kx] = make_float2(ar[k], ai[k]);
+                        const int mx = (N - kx) & (N - 1);
+                        if (mx <= M) base[(N - kyp) * NC + mx] = make_float2(ar[k], -ai[k]);
+                    });
+                } else {
+                    auto untangle = [&](auto Q) {
+                        constexpr int qq = decltype(Q)::value;
+                        static_for<M>([&](auto Kk) {
+                            constexpr int k = decltype(Kk)::value;
+                            constexpr int kp = (qq == 0) ? ((M - k) % M) : (M - 1 - k);
+                            constexpr int kx = 2 * k + qq;
+                            if constexpr (kx <= M) {
+                                const float fr = ar[k], fi = ai[k], gr = ar[kp], gi = ai[kp];
+                                base[kx] = make_float2(0.5f * (fr + gr), 0.5f * (fi - gi));
+                                base[M * NC + kx] = make_float2(0.5f * (fi + gi), 0.5f * (gr - fr));
+                            }
+                        });
+                    };
+                    if (q == 0) untangle(std::integral_constant<int, 0>{});
+                    else        untangle(std::integral_constant<int, 1>{});
+                }
+            }
         }
-    } else {
-        float2* base = reinterpret_cast<float2*>(p.spec_out) +
-                       ((size_t)row * p.C + c0 + g) * (size_t)(N * NC);
-        if (kxp != 0) {
-            static_for<M>([&](auto Kk) {
-                constexpr int k = decltype(Kk)::value;
-                const int ky = 2 * k + q;
-                base[ky * NC + kxp] = make_float2(ar[k], sgn * ai[k]);
-            });
-        } else {
-            auto untangle = [&](auto Q) {
-                constexpr int qq = decltype(Q)::value;
-                static_for<M>([&](auto Kk) {
-                    constexpr int k = decltype(Kk)::value;
-                    constexpr int kp = (qq == 0) ? ((M - k) % M) : (M - 1 - k);
-                    constexpr int ky = 2 * k + qq;
-                    const float fr = ar[k], fi = ai[k], gr = ar[kp], gi = ai[kp];
-                    base[ky * NC] = make_float2(0.5f * (fr + gr), sgn * 0.5f * (fi - gi));
-                    base[ky * NC + M] = make_float2(0.5f * (fi + gi), sgn * 0.5f * (gr - fr));
-                });
-            };
-            if (q == 0) untangle(std::integral_constant<int, 0>{});
-            else        untangle(std::integral_constant<int, 1>{});
+        if constexpr (TMA) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncthreads();
+            if (tid == 0) {
+                // columns beyond the matrix edge (ragged tile) are clipped by the tensor map
+#pragma unroll 1
+                for (int b0 = 0; b0 < 2 * B; b0 += D)
+                    fk_tma_store_3d(&tmS, fk_smem_u32(sStage + (size_t)b0 * G), c0, row, b0);
+                fk_bulk_commit();
+            }
+            store_pending = true;
+        }
+        if (ALIAS) {
+            if (!TMA) __syncthreads();   // step 3 done with the shared buffer before the next tile lands in it
+            const int next = tile + gridDim.x;
+            pending = (next < p.num_tiles) ? stage(next) : false;
+            __syncthreads();
         }
     }
+    if (TMA && store_pending && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------
 // Inverse: half spectra -> cropped, scaled real planes.
 // ---------------------------------------------------------------------------
-template <int N, int G, int LAYOUT>
-__global__ void __launch_bounds__(N* G) c2r_kernel(const FftParams p) {
-    constexpr int T = N * G, NC = N / 2 + 1, M = N / 2, HALF = T / 2;
-    extern __shared__ __align__(16) unsigned char fc_smem[];
-    float* sOut = reinterpret_cast<float*>(fc_smem);
+template <int N, int G, int LAYOUT, int MINB>
+__global__ void __launch_bounds__(N* G, MINB)
+c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
+    constexpr int T = N * G, NC = N / 2 + 1, M = N / 2, HALF = T / 2, B = N * NC;
+    constexpr int PW = MidGeom<N, G>::PW, P = MidGeom<N, G>::P;
+    constexpr bool TMA = (LAYOUT == LAYOUT_FREQ_TMA);
+    constexpr int D = tma_bins_per_box(N);
+    extern __shared__ __align__(128) unsigned char fc_smem[];
     float2* sMid = reinterpret_cast<float2*>(fc_smem);
+    float* sStage = reinterpret_cast<float*>(fc_smem + MidGeom<N, G>::BYTES);
+    __shared__ __align__(8) unsigned long long bar_storage;
+    const uint32_t bar = fk_smem_u32(&bar_storage);
 
     const int tid = threadIdx.x;
-    const int row = blockIdx.x / p.tiles_per_row;
-    const int c0 = (blockIdx.x - row * p.tiles_per_row) * G;
-    const int gcount = min(G, p.C - c0);
-    const int hc = p.h, wc = p.w, wcp = wc | 1, P = p.pitch;
+    const int hc = p.h, wc = p.w, hw = hc * wc;
+    const int gA = tid / wc, cA = tid - gA * wc;                // step 2: (plane, column)
+    const int q = tid / HALF, u = tid - q * HALF;               // step 1: (half, row ky, plane)
+    const int kyp = u / G, gB = u - kyp * G;
+    const bool packed = (kyp == 0);
 
-    // 1. column transforms straight from global memory
-    {
-        const int q = tid / HALF;
-        const int u = tid - q * HALF;
-        const int kxp = u / G;
-        const int g = u - kxp * G;
-        if (g < gcount) {
-            const bool packed = (kxp == 0);
-            const size_t plane = (size_t)p.R * p.ld;
-            const float* fbase = p.spec_in + (size_t)row * p.ld + c0 + g;
-            const float2* bbase = reinterpret_cast<const float2*>(p.spec_in) +
-                                  ((size_t)row * p.C + c0 + g) * (size_t)(N * NC);
-            auto load = [&](int ky) -> float2 {
-                float2 v;
-                if constexpr (LAYOUT == LAYOUT_FREQ_MAJOR) {
-                    const float* a = fbase + (size_t)(ky * NC + kxp) * 2 * plane;
-                    v = make_float2(__ldg(a), __ldg(a + plane));
-                    if (packed) {
-                        const float* b = fbase + (size_t)(ky * NC + M) * 2 * plane;
-                        v.x -= __ldg(b + plane);
-                        v.y += __ldg(b);
-                    }
-                } else {
-                    v = __ldg(bbase + ky * NC + kxp);
-                    if (packed) {
-                        const float2 nq = __ldg(bbase + ky * NC + M);
-                        v.x -= nq.y;
-                        v.y += nq.x;
-                    }
+    auto fetch_tile = [&](int tile) {       // thread 0 only
+        const int row = tile / p.tiles_per_row;
+        const int c0 = (tile - row * p.tiles_per_row) * G;
+        fk_mbar_expect_tx(bar, (uint32_t)(2 * B * G * 4));
+#pragma unroll 1
+        for (int b0 = 0; b0 < 2 * B; b0 += D)
+            fk_tma_load_3d(fk_smem_u32(sStage + (size_t)b0 * G), &tmS, c0, row, b0, bar);
+    };
+    uint32_t phase = 0;
+    if constexpr (TMA) {
+        if (tid == 0) {
+            fk_mbar_init(bar, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            if (blockIdx.x < p.num_tiles) fetch_tile(blockIdx.x);
+        }
+        __syncthreads();
+    }
+
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
+        const int row = tile / p.tiles_per_row;
+        const int c0 = (tile - row * p.tiles_per_row) * G;
+        const int gcount = min(G, p.C - c0);
+
+        // 1. row transforms (along kx): thread = (half q, row kyp, plane gB)
+        float ar[M], ai[M];
+        if constexpr (TMA) {
+            if (!fk_mbar_wait(bar, phase)) return;
+            phase ^= 1u;
+            const float* sb = sStage + kyp * G + gB;
+            auto load = [&](auto Kx) -> float2 {
+                constexpr int kx = decltype(Kx)::value;
+                float2 v = make_float2(sb[kx * NC * G], sb[(B + kx * NC) * G]);
+                if (packed) {       // row ky = N/2 rides as i times itself
+                    v.x -= sb[(B + kx * NC + M) * G];
+                    v.y += sb[(kx * NC + M) * G];
                 }
                 return v;
             };
-            float ar[M], ai[M];
-            auto split = [&](auto Q) {
-                constexpr int qq = decltype(Q)::value;
-                static_for<M>([&](auto J) {
-                    constexpr int j = decltype(J)::value;
-                    const float2 lo = load(j), hi = load(j + M);
-                    if constexpr (qq == 0) {
-                        ar[j] = lo.x + hi.x;
-                        ai[j] = lo.y + hi.y;
+            if (q == 0) load_split<N, true, 0>(load, ar, ai);
+            else        load_split<N, true, 1>(load, ar, ai);
+            __syncthreads();        // staging tile consumed; previous tile's step 2 is done with sMid
+            if (tid == 0 && tile + (int)gridDim.x < p.num_tiles) fetch_tile(tile + gridDim.x);
+        } else {
+            if (gB < gcount) {
+                const size_t mat = (size_t)p.R * p.ld;
+                const float* fbase = p.spec_in + (size_t)kyp * mat + (size_t)row * p.ld + c0 + gB;
+                const float2* bbase = reinterpret_cast<const float2*>(p.spec_in) +
+                                      ((size_t)row * p.C + c0 + gB) * (size_t)(N * NC);
+                auto load = [&](auto Kx) -> float2 {
+                    constexpr int kx = decltype(Kx)::value;
+                    float2 v;
+                    if constexpr (LAYOUT == LAYOUT_FREQ_DIRECT) {
+                        const float* a = fbase + (size_t)(kx * NC) * mat;
+                        v = make_float2(__ldg(a), __ldg(a + (size_t)B * mat));
+                        if (packed) {
+                            v.x -= __ldg(a + (size_t)(B + M) * mat);
+                            v.y += __ldg(a + (size_t)M * mat);
+                        }
                     } else {
-                        const float dr = lo.x - hi.x, di = lo.y - hi.y;
-                        if constexpr (j == 0) {
-                            ar[j] = dr; ai[j] = di;
-                        } else if constexpr (4 * j == N) {
-                            ar[j] = -di; ai[j] = dr;
-                        } else {
-                            constexpr float c = Tw<N, j>::c;
-                            constexpr float s = -Tw<N, j>::s;
-                            ar[j] = fc_fma(s, di, c * dr);
-                            ai[j] = fc_fma(-s, dr, c * di);
+                        auto fetch = [&](int ky) -> float2 {
+                            if (kx <= M) return __ldg(bbase + ky * NC + kx);
+                            float2 t = __ldg(bbase + ((N - ky) & (N - 1)) * NC + (N - kx));
+                            t.y = -t.y;
+                            return t;
+                        };
+                        v = fetch(kyp);
+                        if (packed) {
+                            const float2 nq = fetch(M);
+                            v.x -= nq.y;
+                            v.y += nq.x;
                         }
                     }
-                });
-            };
-            if (q == 0) split(std::integral_constant<int, 0>{});
-            else        split(std::integral_constant<int, 1>{});
-            cfft<M, true>(ar, ai);   // ar/ai[m] = column value at row r = 2m+q
-            float2* dst = sMid + g * P + kxp;
+                    return v;
+                };
+                if (q == 0) load_split<N, true, 0>(load, ar, ai);
+                else        load_split<N, true, 1>(load, ar, ai);
+            }
+            __syncthreads();        // previous tile's step 2 is done with sMid
+        }
+        if (TMA || gB < gcount) {
+            cfft<M, true>(ar, ai);  // ar/ai[m] = value at column c = 2m+q
+            float2* dst = sMid + gB * P + kyp * PW + q;
             static_for<M>([&](auto Mm) {
                 constexpr int m = decltype(Mm)::value;
-                const int r = 2 * m + q;
-                if (r < hc) {
-                    if (!packed) {
-                        dst[r * NC] = make_float2(ar[m], ai[m]);
-                    } else {
-                        dst[r * NC] = make_float2(ar[m], 0.0f);
-                        dst[r * NC + M] = make_float2(ai[m], 0.0f);
-                    }
+                if (!packed) {
+                    dst[2 * m] = make_float2(ar[m], ai[m]);
+                } else {
+                    dst[2 * m] = make_float2(ar[m], 0.0f);
+                    dst[M * PW + 2 * m] = make_float2(ai[m], 0.0f);
                 }
             });
         }
-    }
-    __syncthreads();
+        __syncthreads();
 
-    // 2. row transforms: thread = (plane g, row r), r < hc
-    {
-        const int g = tid / hc, r = tid - g * hc;
-        const bool act = (tid < G * hc) && (g < gcount);
-        float v[N];
-        if (act) {
-            float Xr[NC], Xi[NC];
-            const float2* src = sMid + g * P + r * NC;
-            static_for<NC>([&](auto Kk) {
-                constexpr int k = decltype(Kk)::value;
-                const float2 t = src[k];
-                Xr[k] = t.x; Xi[k] = t.y;
-            });
-            irfft<N>(Xr, Xi, v);
+        // 2. column transforms: thread = (plane gA, column cA), cA < wc; results go straight
+        //    to global memory (lanes run along the row of the plane: contiguous segments)
+        if (gA < gcount) {
+            float v[N];
+            {
+                float Xr[NC], Xi[NC];
+                const float2* src = sMid + gA * P + cA;
+                static_for<NC>([&](auto Kk) {
+                    constexpr int k = decltype(Kk)::value;
+                    const float2 t = src[k * PW];
+                    Xr[k] = t.x; Xi[k] = t.y;
+                });
+                irfft<N>(Xr, Xi, v);
+            }
+            float* dst = p.real_out + ((size_t)row * p.C + c0 + gA) * hw + cA;
+            const float scale = p.scale;
+            if (!p.accumulate) {
+                static_for<N>([&](auto Rr) {
+                    constexpr int r = decltype(Rr)::value;
+                    if (r < hc) dst[r * wc] = v[r] * scale;
+                });
+            } else {
+                static_for<N>([&](auto Rr) {
+                    constexpr int r = decltype(Rr)::value;
+                    if (r < hc) dst[r * wc] = fc_fma(v[r], scale, dst[r * wc]);
+                });
+            }
         }
-        __syncthreads();   // all spectra consumed: reuse the buffer for the real output
-        if (act) {
-            float* dst = sOut + (g * hc + r) * wcp;
-            static_for<N>([&](auto Cc) {
-                constexpr int c = decltype(Cc)::value;
-                if (c < wc) dst[c] = v[c];
-            });
-        }
-    }
-    __syncthreads();
-
-    // 3. coalesced copy-out with scale / accumulate; output planes are contiguous
-    {
-        const long long first = (long long)row * p.C + c0;
-        copy_planes<T, false>(sOut, nullptr, p.real_out + first * hc * wc, gcount,
-                              (long long)hc * wc, hc, wc, wcp, p.scale, p.accumulate);
     }
 }
 
 // ---------------------------------------------------------------------------
 // Host-side launchers.
 // ---------------------------------------------------------------------------
-template <int N>
-struct TileOf;   // planes per CTA for each transform size
-template <> struct TileOf<8>   { static constexpr int G = 32; };
-template <> struct TileOf<16>  { static constexpr int G = 32; };
-template <> struct TileOf<32>  { static constexpr int G = 16; };
-template <> struct TileOf<64>  { static constexpr int G = 8; };
-template <> struct TileOf<128> { static constexpr int G = 2; };
+template <int N> struct FftCfg;   // planes per CTA, buffer aliasing, min CTAs per SM, TMA staging
+template <> struct FftCfg<8>   { static constexpr int G = 32; static constexpr bool ALIAS = false; static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
+template <> struct FftCfg<16>  { static constexpr int G = 16; static constexpr bool ALIAS = false; static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
+template <> struct FftCfg<32>  { static constexpr int G = 8;  static constexpr bool ALIAS = false; static constexpr int MINB = 2, MINB_INV = 3; static constexpr bool TMA = true; };
+template <> struct FftCfg<64>  { static constexpr int G = 4;  static constexpr bool ALIAS = true;  static constexpr int MINB = 2, MINB_INV = 2; static constexpr bool TMA = false; };
+template <> struct FftCfg<128> { static constexpr int G = 2;  static constexpr bool ALIAS = true;  static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = false; };
 
-template <int N, int LAYOUT>
+static inline int fft_sm_count() {
+    static int sms = 0;
+    if (sms == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+            sms = 0;
+    }
+    return sms;
+}
+
+template <class Kern>
+static cudaError_t launch_persistent(Kern kern, int threads, size_t smem, const CUtensorMap& tm,
+                                     FftParams& p, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int per_sm = 0;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
+    if (e != cudaSuccess) return e;
+    const int sms = fft_sm_count();
+    if (per_sm < 1 || sms < 1) return cudaErrorInvalidConfiguration;
+    const long long slots = (long long)per_sm * sms;
+    const int grid = (int)(p.num_tiles < slots ? p.num_tiles : slots);
+    kern<<<grid, threads, smem, st>>>(tm, p);
+    return cudaGetLastError();
+}
+
+// Tensor map of a planar spectrum for the staging tiles: box = G columns x 1 row x D bins.
+template <int N, int G>
+static bool make_spec_map(CUtensorMap* tm, const float* spec, const FftParams& p) {
+    return tc_make_map(tm, spec, N * (N / 2 + 1), p.R, p.C, p.ld, G, 1, CU_TENSOR_MAP_SWIZZLE_NONE,
+                       tma_bins_per_box(N));
+}
+
+template <int N, bool FREQ>
 static cudaError_t launch_r2c_n(FftParams p, cudaStream_t st) {
-    constexpr int G = TileOf<N>::G;
+    using Cfg = FftCfg<N>;
+    constexpr int G = Cfg::G;
+    constexpr int LAYOUT = !FREQ ? LAYOUT_BARE : (Cfg::TMA ? LAYOUT_FREQ_TMA : LAYOUT_FREQ_DIRECT);
     p.tiles_per_row = (p.C + G - 1) / G;
-    p.pitch = smem_plane_pitch(p.h, N, G);
-    const size_t smem = r2c_smem_bytes(N, G, p.h, p.w);
-    auto kern = r2c_kernel<N, G, LAYOUT>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    const long long blocks = (long long)p.R * p.tiles_per_row;
-    if (blocks <= 0 || blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    kern<<<(unsigned)blocks, N * G, smem, st>>>(p);
-    return cudaGetLastError();
+    const long long tiles = (long long)p.R * p.tiles_per_row;
+    if (tiles <= 0 || tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
+    p.num_tiles = (int)tiles;
+    p.in_bytes = real_tile_bytes(G, p.h, p.w);
+    const size_t mid = MidGeom<N, G>::BYTES;
+    size_t smem = Cfg::ALIAS ? (mid > (size_t)p.in_bytes ? mid : (size_t)p.in_bytes)
+                             : mid + (size_t)p.in_bytes;
+    CUtensorMap tm;
+    memset(&tm, 0, sizeof(tm));
+    if (LAYOUT == LAYOUT_FREQ_TMA) {
+        smem += (size_t)2 * N * (N / 2 + 1) * G * sizeof(float);
+        if (!make_spec_map<N, G>(&tm, p.spec_out, p)) return cudaErrorInvalidValue;
+    }
+    return launch_persistent(r2c_kernel<N, G, LAYOUT, Cfg::ALIAS, Cfg::MINB>, N * G, smem, tm, p, st);
 }
 
-template <int N, int LAYOUT>
+template <int N, bool FREQ>
 static cudaError_t launch_c2r_n(FftParams p, cudaStream_t st) {
-    constexpr int G = TileOf<N>::G;
+    using Cfg = FftCfg<N>;
+    constexpr int G = Cfg::G;
+    constexpr int LAYOUT = !FREQ ? LAYOUT_BARE : (Cfg::TMA ? LAYOUT_FREQ_TMA : LAYOUT_FREQ_DIRECT);
     p.tiles_per_row = (p.C + G - 1) / G;
-    p.pitch = smem_plane_pitch(p.h, N, G);
-    const size_t smem = c2r_smem_bytes(N, G, p.h, p.w);
-    auto kern = c2r_kernel<N, G, LAYOUT>;
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    const long long blocks = (long long)p.R * p.tiles_per_row;
-    if (blocks <= 0 || blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
-    kern<<<(unsigned)blocks, N * G, smem, st>>>(p);
-    return cudaGetLastError();
+    const long long tiles = (long long)p.R * p.tiles_per_row;
+    if (tiles <= 0 || tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
+    p.num_tiles = (int)tiles;
+    p.in_bytes = 0;
+    size_t smem = MidGeom<N, G>::BYTES;
+    CUtensorMap tm;
+    memset(&tm, 0, sizeof(tm));
+    if (LAYOUT == LAYOUT_FREQ_TMA) {
+        smem += (size_t)2 * N * (N / 2 + 1) * G * sizeof(float);
+        if (!make_spec_map<N, G>(&tm, p.spec_in, p)) return cudaErrorInvalidValue;
+    }
+    return launch_persistent(c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV>, N * G, smem, tm, p, st);
 }
 
-template <int LAYOUT>
+template <bool FREQ>
 static cudaError_t launch_r2c(int n, const FftParams& p, cudaStream_t st) {
     switch (n) {
-        case 8:   return launch_r2c_n<8, LAYOUT>(p, st);
-        case 16:  return launch_r2c_n<16, LAYOUT>(p, st);
-        case 32:  return launch_r2c_n<32, LAYOUT>(p, st);
-        case 64:  return launch_r2c_n<64, LAYOUT>(p, st);
-        case 128: return launch_r2c_n<128, LAYOUT>(p, st);
+        case 8:   return launch_r2c_n<8, FREQ>(p, st);
+        case 16:  return launch_r2c_n<16, FREQ>(p, st);
+        case 32:  return launch_r2c_n<32, FREQ>(p, st);
+        case 64:  return launch_r2c_n<64, FREQ>(p, st);
+        case 128: return launch_r2c_n<128, FREQ>(p, st);
     }
     return cudaErrorInvalidValue;
 }
-template <int LAYOUT>
+template <bool FREQ>
 static cudaError_t launch_c2r(int n, const FftParams& p, cudaStream_t st) {
     switch (n) {
-        case 8:   return launch_c2r_n<8, LAYOUT>(p, st);
-        case 16:  return launch_c2r_n<16, LAYOUT>(p, st);
-        case 32:  return launch_c2r_n<32, LAYOUT>(p, st);
-        case 64:  return launch_c2r_n<64, LAYOUT>(p, st);
-        case 128: return launch_c2r_n<128, LAYOUT>(p, st);
+        case 8:   return launch_c2r_n<8, FREQ>(p, st);
+        case 16:  return launch_c2r_n<16, FREQ>(p, st);
+        case 32:  return launch_c2r_n<32, FREQ>(p, st);
+        case 64:  return launch_c2r_n<64, FREQ>(p, st);
+        case 128: return launch_c2r_n<128, FREQ>(p, st);
     }
     return cudaErrorInvalidValue;
 }

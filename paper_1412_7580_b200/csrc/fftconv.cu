@@ -27,7 +27,7 @@ constexpr size_t kHeaderBytes = 256;   // workspace header: the device status wo
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int round4(int v) { return (v + 3) & ~3; }
 
-// One frequency-major matrix family: [bins][2][R][ld] floats.
+// One frequency-major matrix family: [2][bins][R][ld] floats (real parts, then imaginary parts).
 struct SpecDesc {
     int R, C, ld;
     size_t bytes(int bins) const { return (size_t)bins * 2 * R * ld * sizeof(float); }
@@ -131,9 +131,8 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         fp.real_in = in; fp.spec_out = spec;
         fp.h = o.h; fp.w = o.w;
         fp.R = o.spec.R; fp.C = o.spec.C; fp.ld = o.spec.ld;
-        fp.in_rs = o.spec.C; fp.in_cs = 1; fp.conj = 0;
         g_launches.fetch_add(1, std::memory_order_relaxed);
-        return fc::launch_r2c<fc::LAYOUT_FREQ_MAJOR>(plan->n, fp, st);
+        return fc::launch_r2c<true>(plan->n, fp, st);
     };
     const bool timing = plan->timing && plan->ev_made;
     auto mark = [&](int i) { if (timing) cudaEventRecord(plan->ev[i], st); };
@@ -162,7 +161,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     ip.scale = 1.0f / ((float)plan->n * (float)plan->n);
     ip.accumulate = accumulate ? 1 : 0;
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    if (fc::launch_c2r<fc::LAYOUT_FREQ_MAJOR>(plan->n, ip, st) != cudaSuccess) return FFTCONV_ECUDA;
+    if (fc::launch_c2r<true>(plan->n, ip, st) != cudaSuccess) return FFTCONV_ECUDA;
     mark(4);
     if (timing) plan->timed = true;
     return FFTCONV_OK;
@@ -302,9 +301,8 @@ FFTCONV_API int fft2d_r2c(const float* in, void* out_c, int batch, int h, int w,
     fc::FftParams p{};
     p.real_in = in; p.spec_out = static_cast<float*>(out_c);
     p.h = h; p.w = w; p.R = 1; p.C = batch; p.ld = batch;
-    p.in_rs = 0; p.in_cs = 1; p.conj = 0;
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return fc::launch_r2c<fc::LAYOUT_BARE>(n, p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+    return fc::launch_r2c<false>(n, p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
                ? FFTCONV_OK : FFTCONV_ECUDA;
 }
 
@@ -318,7 +316,7 @@ FFTCONV_API int fft2d_c2r(const void* in_c, float* out, int batch, int n, int oh
     p.h = oh; p.w = ow; p.R = 1; p.C = batch; p.ld = batch;
     p.scale = scale; p.accumulate = accumulate ? 1 : 0;
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return fc::launch_c2r<fc::LAYOUT_BARE>(n, p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+    return fc::launch_c2r<false>(n, p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
                ? FFTCONV_OK : FFTCONV_ECUDA;
 }
 

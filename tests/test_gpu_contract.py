@@ -17,29 +17,29 @@ def run(bins, M, N, K, math, seed=0, transA=False, transB=False, conjA=False, co
 
     def operand(rows, trans, fill):
         """Logical [bins][rows][K] complex matrix, stored planar either as
-        [bins][2][rows][ld>=K] or, transposed, as [bins][2][K][ld>=rows]."""
+        [2][bins][rows][ld>=K] or, transposed, as [2][bins][K][ld>=rows]."""
         re = rng.standard_normal((bins, rows, K), dtype=np.float32)
         im = rng.standard_normal((bins, rows, K), dtype=np.float32)
         if not trans:
-            buf = np.full((bins, 2, rows, r4(K)), fill, np.float32)   # padding must never be read as data
-            buf[:, 0, :, :K], buf[:, 1, :, :K] = re, im
+            buf = np.full((2, bins, rows, r4(K)), fill, np.float32)   # padding must never be read as data
+            buf[0, :, :, :K], buf[1, :, :, :K] = re, im
         else:
-            buf = np.full((bins, 2, K, r4(rows)), fill, np.float32)
-            buf[:, 0, :, :rows], buf[:, 1, :, :rows] = re.transpose(0, 2, 1), im.transpose(0, 2, 1)
+            buf = np.full((2, bins, K, r4(rows)), fill, np.float32)
+            buf[0, :, :, :rows], buf[1, :, :, :rows] = re.transpose(0, 2, 1), im.transpose(0, 2, 1)
         return buf, re.astype(np.float64) + 1j * im.astype(np.float64)
 
     A, Ac = operand(M, transA, 1e30)
     B, Bc = operand(N, transB, -1e30)
     ldc = r4(N)
     Ad, Bd = torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda()
-    Cd = torch.full((bins, 2, M, ldc), float("nan"), device="cuda")
+    Cd = torch.full((2, bins, M, ldc), float("nan"), device="cuda")
     status = torch.zeros(64, dtype=torch.int32, device="cuda")
     fc.fftconv_bin_contract(Ad, Bd, Cd, M, N, K, transA, transB, conjA, conjB, math=math,
                             status_word=status)
     torch.cuda.synchronize()
     assert int(status[0].item()) == 0
     C = Cd.cpu().numpy().astype(np.float64)
-    got = C[:, 0, :, :N] + 1j * C[:, 1, :, :N]
+    got = C[0, :, :, :N] + 1j * C[1, :, :, :N]
     ref = oracle.bin_contract(Ac, Bc, conjA, conjB)
     assert np.all(np.isfinite(got.real)) and np.all(np.isfinite(got.imag))
     # padding columns of C (N..ldc-1) are scratch: untouched or zero, never data
