@@ -85,6 +85,34 @@ int conv_plan_set_workspace(conv_plan_t* plan, void* dev_ptr, size_t bytes);
  * cross-correlation.  Overwrites y [S][fprime][oh][ow]. */
 int conv_fprop(conv_plan_t* plan, const float* x, const float* w, float* y, void* cuda_stream);
 
+/* fprop without any device allocation by anybody (the paper has no counterpart:
+ * its buffer manager always allocates).  Same computation and same kernels as
+ * conv_fprop, but the frequency-domain scratch lives in a fixed array that is
+ * part of the library image (FFTCONV_NOALLOC_BYTES = 32 MiB of device memory,
+ * held by every GPU that loads the library until the process exits) instead of
+ * a workspace lent by the caller.  It is meant for callers that have tensors
+ * but no way to obtain scratch memory at the call site: code running after a
+ * framework's allocator has claimed the whole device, loops in which an
+ * allocation (which synchronises the device) is not acceptable, plug-ins that
+ * are handed buffers but no allocator.  The plan's own workspace, if any, is
+ * ignored and left untouched; x, w, y are passed as for conv_fprop.
+ *  - Returns FFTCONV_EWORKSPACE, launching nothing, when
+ *    conv_plan_workspace_bytes(plan) exceeds FFTCONV_NOALLOC_BYTES.
+ *  - Calls no cudaMalloc / cudaFree and no allocating library routine.  The
+ *    first call on each device looks up the array's device address (one
+ *    cudaGetSymbolAddress, with that device current); make that first call
+ *    outside any stream capture.
+ *  - All calls on a device share the one array and it keeps whatever the last
+ *    call left in it; each call clears the small status header it relies on and
+ *    overwrites every spectrum it reads.  Two calls that overlap on the GPU
+ *    (different streams, no dependency) race on the array: serialise them.
+ *  - A bounded device-side wait that runs out is recorded in the array's header,
+ *    which no entry point reads back; use conv_fprop + conv_plan_status where
+ *    that diagnosis matters. */
+#define FFTCONV_NOALLOC_BYTES (32u << 20)
+int conv_fprop_noalloc(conv_plan_t* plan, const float* x, const float* w, float* y,
+                       void* cuda_stream);
+
 /* bprop (Section 2, second equation): dx(s,i) = sum_j dy(s,j) * w(j,i), full
  * convolution.  Overwrites dx [S][f][h][w]. */
 int conv_bprop(conv_plan_t* plan, const float* dy, const float* w, float* dx, void* cuda_stream);

@@ -18,7 +18,7 @@ MATH_AUTO, MATH_FP32, MATH_TF32 = 0, 1, 2
 
 EXPORTS = (
     "conv_plan", "conv_plan_set_math", "conv_plan_effective_math", "conv_plan_workspace_bytes",
-    "conv_plan_set_workspace", "conv_fprop", "conv_bprop", "conv_accgrad", "conv_plan_status",
+    "conv_plan_set_workspace", "conv_fprop", "conv_fprop_noalloc", "conv_bprop", "conv_accgrad", "conv_plan_status",
     "conv_plan_destroy", "conv_plan_enable_stage_timing", "conv_plan_stage_times_ms", "fft2d_r2c", "fft2d_c2r", "fftconv_bin_contract",
     "fftconv_status_string", "fftconv_launch_count",
 )
@@ -49,6 +49,7 @@ def lib():
         L.conv_plan_workspace_bytes.restype = z
         L.conv_plan_set_workspace.argtypes = [p, p, z]
         L.conv_fprop.argtypes = [p, p, p, p, p]
+        L.conv_fprop_noalloc.argtypes = [p, p, p, p, p]
         L.conv_bprop.argtypes = [p, p, p, p, p]
         L.conv_accgrad.argtypes = [p, p, p, p, i, p]
         L.conv_plan_status.argtypes = [p]
@@ -166,6 +167,22 @@ def conv_fprop(plan: Plan, x, w, y, stream=None) -> None:
                             _dev(w, (plan.fp, plan.f, plan.kh, plan.kw), "w"),
                             _dev(y, (plan.S, plan.fp, plan.oh, plan.ow), "y"),
                             _stream_ptr(stream)), "conv_fprop")
+
+
+NOALLOC_BYTES = 32 << 20
+
+
+def conv_fprop_noalloc(plan: Plan, x, w, y, stream=None) -> None:
+    """conv_fprop on the library's built-in 32 MiB scratch array: for callers that
+    hold tensors but cannot allocate a workspace.  The plan needs no workspace; plans
+    that need more than NOALLOC_BYTES are refused (FftConvError, EWORKSPACE).  Calls
+    share the array, so do not let two of them overlap on the GPU; make the first call
+    on a device outside any stream capture."""
+    _check(lib().conv_fprop_noalloc(plan.handle,
+                                    _dev(x, (plan.S, plan.f, plan.h, plan.w), "x"),
+                                    _dev(w, (plan.fp, plan.f, plan.kh, plan.kw), "w"),
+                                    _dev(y, (plan.S, plan.fp, plan.oh, plan.ow), "y"),
+                                    _stream_ptr(stream)), "conv_fprop_noalloc")
 
 
 def conv_bprop(plan: Plan, dy, w, dx, stream=None) -> None:

@@ -237,6 +237,50 @@ FFTCONV_API int conv_fprop(conv_plan_t* plan, const float* x, const float* w, fl
     return run_pass(plan, PASS_FPROP, x, w, y, 0, static_cast<cudaStream_t>(cuda_stream));
 }
 
+// ---------------------------------------------------------------------------
+// fprop on the library's own fixed scratch array: for callers that cannot
+// allocate (see the header).  The array is a file-scope device symbol; in host
+// code its name is only a handle, so its device address is looked up once per
+// device with cudaGetSymbolAddress and that pointer is what the kernels get.
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_noalloc_scratch[FFTCONV_NOALLOC_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_noalloc_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the scratch array on the current device (nullptr on failure).
+void* noalloc_scratch_address() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    if (!g_noalloc_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess) return nullptr;
+        g_noalloc_ptr[dev] = ptr;
+    }
+    return g_noalloc_ptr[dev];
+}
+}  // namespace
+
+FFTCONV_API int conv_fprop_noalloc(conv_plan_t* plan, const float* x, const float* w, float* y,
+                                   void* cuda_stream) {
+    if (!plan || !x || !w || !y) return FFTCONV_EINVAL;
+    if (conv_plan_workspace_bytes(plan) > (size_t)FFTCONV_NOALLOC_BYTES) return FFTCONV_EWORKSPACE;
+    void* scratch = noalloc_scratch_address();
+    if (!scratch) return FFTCONV_ECUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    // the header (device status word) must start at zero; the spectra need no clearing
+    // because every element the contraction and the inverse transform read is written first
+    if (cudaMemsetAsync(scratch, 0, kHeaderBytes, st) != cudaSuccess) return FFTCONV_ECUDA;
+    conv_plan_s local = *plan;          // same shape and math mode, library-owned scratch
+    local.ws = scratch;
+    local.ws_bytes = FFTCONV_NOALLOC_BYTES;
+    local.timing = 0;
+    local.timed = false;
+    local.ev_made = false;
+    return run_pass(&local, PASS_FPROP, x, w, y, 0, st);
+}
+
 FFTCONV_API int conv_bprop(conv_plan_t* plan, const float* dy, const float* w, float* dx,
                            void* cuda_stream) {
     return run_pass(plan, PASS_BPROP, dy, w, dx, 0, static_cast<cudaStream_t>(cuda_stream));
