@@ -155,3 +155,11 @@ def sample_coords(dims, count: int, seed: int) -> np.ndarray:
     rnd = np.stack([rng.integers(0, d, size=max(count - 16, 0)) for d in dims], axis=1)
     out = np.concatenate([corners, rnd], axis=0)[:max(count, 1)]
     return np.ascontiguousarray(out, dtype=np.int32)
+
+
+def shard_range(S: int, rank: int, world: int):
+    """Contiguous slice [lo, hi) of the minibatch owned by `rank` when S samples are
+    split over `world` data-parallel ranks (sizes differ by at most one)."""
+    base, extra = divmod(int(S), int(world))
+    lo = rank * base + min(rank, extra)
+    return lo, lo + base + (1 if rank < extra else 0)
