@@ -272,8 +272,8 @@ def run_ours(args, s):
         step(); reps += 1
     torch.cuda.synchronize()
     t1 = time.time()
-    launches = 12 * args.steps
-    assert fc.fftconv_launch_count() - launches0 == 12 * (args.steps + reps)
+    launches = 9 * args.steps          # per pass: both forward FFTs (one launch), contraction, inverse FFT
+    assert fc.fftconv_launch_count() - launches0 == 9 * (args.steps + reps)
     clocks = sampler.stop(t0, t1) if rank == 0 else None
     ms_step = ms_total / args.steps
 

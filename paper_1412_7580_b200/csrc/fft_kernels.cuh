@@ -177,14 +177,24 @@ __device__ __forceinline__ void load_split(Load&& load, float (&ar)[N / 2], floa
     });
 }
 
+#ifdef FC_EXP_TIMELINE
+__device__ long long fc_timeline[16];
+#define FC_TICK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { long long t_ = clock64(); fc_timeline[i] += t_ - tl_last; tl_last = t_; } } while (0)
+#else
+#define FC_TICK(i) do { } while (0)
+#endif
+
 // ---------------------------------------------------------------------------
 // Forward: real planes -> half spectra.
 // ALIAS: the half-spectrum scratch overwrites the staging area of the real tile
 // (no prefetch of the next tile); used where one tile nearly fills shared memory.
 // ---------------------------------------------------------------------------
-template <int N, int G, int LAYOUT, bool ALIAS, int MINB>
+template <int N, int G, int LAYOUT, bool ALIAS, bool SALIAS, int MINB>
 __global__ void __launch_bounds__(N* G, MINB)
-r2c_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
+r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUtensorMap tmS1,
+           const FftParams p0, const FftParams p1) {
+    // Two operands can share one launch (both forward transforms of a pass): tiles
+    // [0, p0.num_tiles) belong to the first, the rest to the second.
     constexpr int T = N * G, NC = N / 2 + 1, M = N / 2, HALF = T / 2, B = N * NC;
     constexpr int PW = MidGeom<N, G>::PW, P = MidGeom<N, G>::P;
     constexpr bool TMA = (LAYOUT == LAYOUT_FREQ_TMA);
@@ -192,42 +202,71 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
     static_assert(HALF % 32 == 0, "the two halves of a row transform must be warp-uniform");
     extern __shared__ __align__(128) unsigned char fc_smem[];
     float* sIn = reinterpret_cast<float*>(fc_smem);
-    unsigned char* mid_base = fc_smem + (ALIAS ? 0 : p.in_bytes);
+    unsigned char* mid_base = fc_smem + (ALIAS ? 0 : p0.in_bytes);
     float2* sMid = reinterpret_cast<float2*>(mid_base);
+    // SALIAS: the staging tile reuses the scratch (one more barrier per tile, a third less
+    // shared memory, so more CTAs stay resident)
     float* sStage = reinterpret_cast<float*>(
-        mid_base + (ALIAS ? (p.in_bytes > MidGeom<N, G>::BYTES ? p.in_bytes : MidGeom<N, G>::BYTES)
-                          : MidGeom<N, G>::BYTES));
+        SALIAS ? mid_base
+               : mid_base + (ALIAS ? (p0.in_bytes > MidGeom<N, G>::BYTES ? p0.in_bytes : MidGeom<N, G>::BYTES)
+                                   : MidGeom<N, G>::BYTES));
     __shared__ __align__(8) unsigned long long bar_storage;
     const uint32_t bar = fk_smem_u32(&bar_storage);
 
     const int tid = threadIdx.x;
-    const int h = p.h, w = p.w, hw = h * w;
-    // thread roles, fixed for the whole kernel
-    const int gA = tid / w, cA = tid - gA * w;                  // step 2: (plane, column)
-    const int q = tid / HALF, u = tid - q * HALF;               // step 3: (half, row ky, plane)
+    const int total_tiles = p0.num_tiles + p1.num_tiles;
+    // thread roles of step 3, fixed for the whole kernel: (half, row ky, plane)
+    const int q = tid / HALF, u = tid - q * HALF;
     const int kyp = u / G, gB = u - kyp * G;
+    const int q4 = tid / (T / 4), u4 = tid - q4 * (T / 4);      // step 2, narrow planes: quarter
+    // operand-dependent state, set by select()
+    int h, w, hw, opC;
+    int gA, cA, g4, c4;                                         // step 2: (plane, column)
+    bool split4;                                                // narrow planes: 4 threads per column
+    auto select = [&](bool second) {
+        h = second ? p1.h : p0.h;
+        w = second ? p1.w : p0.w;
+        opC = second ? p1.C : p0.C;
+        hw = h * w;
+        gA = tid / w; cA = tid - gA * w;
+        split4 = (4 * G * w <= T);
+        g4 = u4 / w; c4 = u4 - g4 * w;
+    };
+    // tile index -> (operand, row, tile in row)
+    auto locate = [&](int tile, bool& second, int& row, int& tcol) {
+        second = tile >= p0.num_tiles;
+        const int t = second ? tile - p0.num_tiles : tile;
+        const int tpr = second ? p1.tiles_per_row : p0.tiles_per_row;
+        row = t / tpr;
+        tcol = t - row * tpr;
+    };
 
     if (tid == 0) {
         fk_mbar_init(bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (!ALIAS) {
-        // columns >= w of the scratch are never written: zero them once, read them freely
-        for (int i = tid; i < G * P; i += T) sMid[i] = make_float2(0.0f, 0.0f);
-    }
     __syncthreads();
 
-    // Stage the planes of `tile`.  Returns true if the copy is asynchronous (wait on the
+    // Side jobs are spread over different warps so that no single thread strings them
+    // together: thread T/2 issues the input copy, the last warp issues the TMA stores.
+    constexpr int NB = 2 * B / D;                       // TMA boxes per tile
+    static_assert(!TMA || NB <= 32, "one lane per TMA box");
+    const bool is_loader = (tid == T / 2);
+    const bool is_storer = (tid >= T - 32) && ((tid & 31) < NB);
+
+    // Stage the planes of a tile.  Returns true if the copy is asynchronous (wait on the
     // barrier before reading), false if it was done with plain loads by all threads.
-    auto stage = [&](int tile) -> bool {
-        const int row = tile / p.tiles_per_row;
-        const int c0 = (tile - row * p.tiles_per_row) * G;
-        const int gcount = min(G, p.C - c0);
-        const float* src = p.real_in + ((size_t)row * p.C + c0) * hw;
-        const int total = gcount * hw;
+    auto stage = [&](bool second, int row, int tcol) -> bool {
+        const int sh = second ? p1.h : p0.h, sw = second ? p1.w : p0.w;
+        const int sC = second ? p1.C : p0.C;
+        const float* base = second ? p1.real_in : p0.real_in;
+        const int c0 = tcol * G;
+        const int gcount = min(G, sC - c0);
+        const float* src = base + ((size_t)row * sC + c0) * (sh * sw);
+        const int total = gcount * sh * sw;
         if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
             const int bulk = total & ~3;
-            if (tid == 0 && bulk > 0) {
+            if (is_loader && bulk > 0) {
                 fk_mbar_expect_tx(bar, (uint32_t)bulk * 4u);
                 fk_bulk_g2s(fk_smem_u32(sIn), src, (uint32_t)bulk * 4u, bar);
             }
@@ -240,45 +279,112 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
 
     uint32_t phase = 0;
     bool pending = false, store_pending = false;
-    if (blockIdx.x < p.num_tiles) pending = stage(blockIdx.x);
+    bool second = false, second_n = false;
+    int row = 0, tcol = 0, row_n = 0, tcol_n = 0;
+    if ((int)blockIdx.x < total_tiles) {
+        locate(blockIdx.x, second_n, row_n, tcol_n);
+        pending = stage(second_n, row_n, tcol_n);
+    }
     __syncthreads();           // plain-load parts of the first tile are visible to everyone
 
-    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-        const int row = tile / p.tiles_per_row;
-        const int c0 = (tile - row * p.tiles_per_row) * G;
-        const int gcount = min(G, p.C - c0);
+#ifdef FC_EXP_TIMELINE
+    long long tl_last = clock64();
+#endif
+    for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        second = second_n; row = row_n; tcol = tcol_n;
+        select(second);
+        const FftParams& p = second ? p1 : p0;
+        const CUtensorMap* tmS = second ? &tmS1 : &tmS0;
+        const int c0 = tcol * G;
+        const int gcount = min(G, opC - c0);
+        const int next = tile + gridDim.x;
+        if (next < total_tiles) locate(next, second_n, row_n, tcol_n);
 
+        FC_TICK(0);
         if (pending) {
             if (!fk_mbar_wait(bar, phase)) return;     // copy never landed: give up
             phase ^= 1u;
         }
+        FC_TICK(1);
 
-        // 2. column transforms: thread = (plane gA, column cA), cA < w
+        // 2. column transforms.  Wide planes: thread = (plane gA, column cA), cA < w, one real
+        //    FFT of length N each.  Narrow planes (filters): four threads per column, thread
+        //    q4 computing the outputs ky = 4k + q4 through one radix-4 decimation-in-frequency
+        //    step and a complex FFT of length N/4, so that the few columns still occupy the CTA.
         {
-            const bool act = (gA < gcount);             // gA < G follows from tid < G*w
+            constexpr int L = N / 4;
             float Xr[NC], Xi[NC];
-            if (act) {
-                float v[N];
-                const float* src = sIn + gA * hw + cA;
-                static_for<N>([&](auto Rr) {
-                    constexpr int r = decltype(Rr)::value;
-                    v[r] = (r < h) ? src[r * w] : 0.0f;
-                });
-                rfft<N>(v, Xr, Xi);
+            float br[L], bi[L];
+            bool act;
+            if (!split4) {
+                act = (gA < gcount);                    // gA < G follows from tid < G*w
+                if (act) {
+                    float v[N];
+                    const float* src = sIn + gA * hw + cA;
+                    static_for<N>([&](auto Rr) {
+                        constexpr int r = decltype(Rr)::value;
+                        v[r] = (r < h) ? src[r * w] : 0.0f;
+                    });
+                    rfft<N>(v, Xr, Xi);
+                }
+            } else {
+                act = (u4 < G * w) && (g4 < gcount);
+                if (act) {
+                    const float* src = sIn + g4 * hw + c4;
+                    auto quarter = [&](auto Q) {
+                        constexpr int qq = decltype(Q)::value;
+                        static_for<L>([&](auto J) {
+                            constexpr int j = decltype(J)::value;
+                            const float x0 = (j < h) ? src[j * w] : 0.0f;
+                            const float x1 = (j + L < h) ? src[(j + L) * w] : 0.0f;
+                            const float x2 = (j + 2 * L < h) ? src[(j + 2 * L) * w] : 0.0f;
+                            const float x3 = (j + 3 * L < h) ? src[(j + 3 * L) * w] : 0.0f;
+                            if constexpr (qq == 0) {
+                                br[j] = (x0 + x2) + (x1 + x3); bi[j] = 0.0f;
+                            } else if constexpr (qq == 2) {
+                                const float t = (x0 + x2) - (x1 + x3);
+                                br[j] = t * Tw<N, 2 * j>::c; bi[j] = -t * Tw<N, 2 * j>::s;
+                            } else {
+                                // d = (x0 - x2) -+ i (x1 - x3), times w_N^(qq j) = (c, -s)
+                                const float dr = x0 - x2, di = (qq == 1) ? (x3 - x1) : (x1 - x3);
+                                constexpr float c = Tw<N, qq * j>::c, sn = Tw<N, qq * j>::s;
+                                br[j] = fc_fma(sn, di, c * dr);
+                                bi[j] = fc_fma(-sn, dr, c * di);
+                            }
+                        });
+                    };
+                    if (q4 == 0) quarter(std::integral_constant<int, 0>{});
+                    else if (q4 == 1) quarter(std::integral_constant<int, 1>{});
+                    else if (q4 == 2) quarter(std::integral_constant<int, 2>{});
+                    else quarter(std::integral_constant<int, 3>{});
+                    cfft<L, false>(br, bi);             // br/bi[k] = X[ky = 4k + q4]
+                }
             }
-            if (TMA && store_pending && tid == 0) fk_bulk_wait_read();   // staging tile free again
+            FC_TICK(2);
+            if (TMA && store_pending && is_storer) fk_bulk_wait_read();  // staging tile free again
+            FC_TICK(3);
             __syncthreads();   // tile consumed (and the previous tile's step 3 is done with sMid)
-            const int next = tile + gridDim.x;
-            if (!ALIAS) pending = (next < p.num_tiles) ? stage(next) : false;
+            FC_TICK(4);
+            if (!ALIAS) pending = (next < total_tiles) ? stage(second_n, row_n, tcol_n) : false;
             if (act) {
-                float2* dst = sMid + gA * P + cA;
-                static_for<NC>([&](auto Kk) {
-                    constexpr int k = decltype(Kk)::value;
-                    dst[k * PW] = make_float2(Xr[k], Xi[k]);
-                });
+                if (!split4) {
+                    float2* dst = sMid + gA * P + cA;
+                    static_for<NC>([&](auto Kk) {
+                        constexpr int k = decltype(Kk)::value;
+                        dst[k * PW] = make_float2(Xr[k], Xi[k]);
+                    });
+                } else {
+                    float2* dst = sMid + g4 * P + c4 + q4 * PW;
+                    static_for<L>([&](auto Kk) {
+                        constexpr int k = decltype(Kk)::value;
+                        if (4 * k + q4 <= M) dst[4 * k * PW] = make_float2(br[k], bi[k]);
+                    });
+                }
             }
         }
+        FC_TICK(5);
         __syncthreads();
+        FC_TICK(6);
 
         // 3. row transforms: thread = (half q, row kyp, plane gB)
         if (TMA || gB < gcount) {
@@ -288,16 +394,18 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             auto load = [&](auto Cc) -> float2 {
                 constexpr int c = decltype(Cc)::value;
                 float2 v;
-                if constexpr (ALIAS) {
-                    if (c >= w) return make_float2(0.0f, 0.0f);
-                }
+                if (c >= w) return make_float2(0.0f, 0.0f);   // columns the tile never wrote
                 v = rowp[c];
                 if (packed) v.y = rowp[M * PW + c].x;   // row ky = N/2 rides as the imaginary part
                 return v;
             };
             if (q == 0) load_split<N, false, 0>(load, ar, ai);
             else        load_split<N, false, 1>(load, ar, ai);
+            FC_TICK(7);
+            if constexpr (TMA && SALIAS) __syncthreads();   // scratch consumed: it becomes the staging tile
+            FC_TICK(8);
             cfft<M, false>(ar, ai);                     // ar/ai[k] = F[kx = 2k+q]
+            FC_TICK(9);
 
             if constexpr (LAYOUT != LAYOUT_BARE) {
                 // element (part, bin = kx*NC + ky, plane g): staging offset (part*B + bin)*G + g,
@@ -367,26 +475,29 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
                 }
             }
         }
+        FC_TICK(10);
         if constexpr (TMA) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            FC_TICK(11);
             __syncthreads();
-            if (tid == 0) {
-                // columns beyond the matrix edge (ragged tile) are clipped by the tensor map
-#pragma unroll 1
-                for (int b0 = 0; b0 < 2 * B; b0 += D)
-                    fk_tma_store_3d(&tmS, fk_smem_u32(sStage + (size_t)b0 * G), c0, row, b0);
+            FC_TICK(12);
+            if (is_storer) {
+                // one box per lane; columns beyond the matrix edge (ragged tile) are clipped
+                // by the tensor map
+                const int b0 = (tid & 31) * D;
+                fk_tma_store_3d(tmS, fk_smem_u32(sStage + (size_t)b0 * G), c0, row, b0);
                 fk_bulk_commit();
             }
             store_pending = true;
+            FC_TICK(13);
         }
         if (ALIAS) {
             if (!TMA) __syncthreads();   // step 3 done with the shared buffer before the next tile lands in it
-            const int next = tile + gridDim.x;
-            pending = (next < p.num_tiles) ? stage(next) : false;
+            pending = (next < total_tiles) ? stage(second_n, row_n, tcol_n) : false;
             __syncthreads();
         }
     }
-    if (TMA && store_pending && tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if (TMA && store_pending && is_storer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------
@@ -412,28 +523,40 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
     const int kyp = u / G, gB = u - kyp * G;
     const bool packed = (kyp == 0);
 
-    auto fetch_tile = [&](int tile) {       // thread 0 only
-        const int row = tile / p.tiles_per_row;
-        const int c0 = (tile - row * p.tiles_per_row) * G;
-        fk_mbar_expect_tx(bar, (uint32_t)(2 * B * G * 4));
-#pragma unroll 1
-        for (int b0 = 0; b0 < 2 * B; b0 += D)
-            fk_tma_load_3d(fk_smem_u32(sStage + (size_t)b0 * G), &tmS, c0, row, b0, bar);
+    const int tpr = p.tiles_per_row;
+    const int step_rows = gridDim.x / tpr, step_cols = gridDim.x - step_rows * tpr;
+    auto advance = [&](int& row, int& tcol) {
+        row += step_rows; tcol += step_cols;
+        if (tcol >= tpr) { tcol -= tpr; ++row; }
+    };
+    // the last warp fetches the spectrum tiles: lane 0 arms the barrier, one TMA box per lane
+    constexpr int NB = 2 * B / D;
+    static_assert(!TMA || NB <= 32, "one lane per TMA box");
+    const bool is_fetcher = (tid >= T - 32);
+    auto fetch_tile = [&](int row, int tcol) {      // called by the whole last warp
+        if ((tid & 31) == 0) fk_mbar_expect_tx(bar, (uint32_t)(2 * B * G * 4));
+        __syncwarp();
+        if ((tid & 31) < NB) {
+            const int b0 = (tid & 31) * D;
+            fk_tma_load_3d(fk_smem_u32(sStage + (size_t)b0 * G), &tmS, tcol * G, row, b0, bar);
+        }
     };
     uint32_t phase = 0;
+    int row = blockIdx.x / tpr, tcol = blockIdx.x - (blockIdx.x / tpr) * tpr;
     if constexpr (TMA) {
         if (tid == 0) {
             fk_mbar_init(bar, 1);
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            if (blockIdx.x < p.num_tiles) fetch_tile(blockIdx.x);
         }
         __syncthreads();
+        if (is_fetcher && blockIdx.x < p.num_tiles) fetch_tile(row, tcol);
     }
 
-    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
-        const int row = tile / p.tiles_per_row;
-        const int c0 = (tile - row * p.tiles_per_row) * G;
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, advance(row, tcol)) {
+        const int c0 = tcol * G;
         const int gcount = min(G, p.C - c0);
+        int row_n = row, tcol_n = tcol;
+        advance(row_n, tcol_n);
 
         // 1. row transforms (along kx): thread = (half q, row kyp, plane gB)
         float ar[M], ai[M];
@@ -453,7 +576,7 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             if (q == 0) load_split<N, true, 0>(load, ar, ai);
             else        load_split<N, true, 1>(load, ar, ai);
             __syncthreads();        // staging tile consumed; previous tile's step 2 is done with sMid
-            if (tid == 0 && tile + (int)gridDim.x < p.num_tiles) fetch_tile(tile + gridDim.x);
+            if (is_fetcher && tile + (int)gridDim.x < p.num_tiles) fetch_tile(row_n, tcol_n);
         } else {
             if (gB < gcount) {
                 const size_t mat = (size_t)p.R * p.ld;
@@ -541,11 +664,11 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
 // Host-side launchers.
 // ---------------------------------------------------------------------------
 template <int N> struct FftCfg;   // planes per CTA, buffer aliasing, min CTAs per SM, TMA staging
-template <> struct FftCfg<8>   { static constexpr int G = 32; static constexpr bool ALIAS = false; static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
-template <> struct FftCfg<16>  { static constexpr int G = 16; static constexpr bool ALIAS = false; static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
-template <> struct FftCfg<32>  { static constexpr int G = 8;  static constexpr bool ALIAS = false; static constexpr int MINB = 2, MINB_INV = 3; static constexpr bool TMA = true; };
-template <> struct FftCfg<64>  { static constexpr int G = 4;  static constexpr bool ALIAS = false; static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = true; };
-template <> struct FftCfg<128> { static constexpr int G = 2;  static constexpr bool ALIAS = true;  static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = false; };
+template <> struct FftCfg<8>   { static constexpr int G = 32; static constexpr bool ALIAS = false, SALIAS = true;  static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
+template <> struct FftCfg<16>  { static constexpr int G = 16; static constexpr bool ALIAS = false, SALIAS = true;  static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
+template <> struct FftCfg<32>  { static constexpr int G = 8;  static constexpr bool ALIAS = false, SALIAS = true;  static constexpr int MINB = 3, MINB_INV = 3; static constexpr bool TMA = true; };
+template <> struct FftCfg<64>  { static constexpr int G = 4;  static constexpr bool ALIAS = false, SALIAS = false; static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = true; };
+template <> struct FftCfg<128> { static constexpr int G = 2;  static constexpr bool ALIAS = true,  SALIAS = false; static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = false; };
 
 static inline int fft_sm_count() {
     static int sms = 0;
@@ -558,9 +681,8 @@ static inline int fft_sm_count() {
     return sms;
 }
 
-template <class Kern>
-static cudaError_t launch_persistent(Kern kern, int threads, size_t smem, const CUtensorMap& tm,
-                                     FftParams& p, cudaStream_t st) {
+static cudaError_t persistent_grid(const void* kern, int threads, size_t smem, long long tiles,
+                                   int* grid) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     int per_sm = 0;
@@ -569,9 +691,8 @@ static cudaError_t launch_persistent(Kern kern, int threads, size_t smem, const 
     const int sms = fft_sm_count();
     if (per_sm < 1 || sms < 1) return cudaErrorInvalidConfiguration;
     const long long slots = (long long)per_sm * sms;
-    const int grid = (int)(p.num_tiles < slots ? p.num_tiles : slots);
-    kern<<<grid, threads, smem, st>>>(tm, p);
-    return cudaGetLastError();
+    *grid = (int)(tiles < slots ? tiles : slots);
+    return cudaSuccess;
 }
 
 // Tensor map of a planar spectrum for the staging tiles: box = G columns x 1 row x D bins.
@@ -581,26 +702,51 @@ static bool make_spec_map(CUtensorMap* tm, const float* spec, const FftParams& p
                        tma_bins_per_box(N));
 }
 
+template <int G>
+static bool fill_tiling(FftParams& p) {
+    p.tiles_per_row = (p.C + G - 1) / G;
+    const long long tiles = (long long)p.R * p.tiles_per_row;
+    if (tiles <= 0 || tiles > 0x3fffffffLL) return false;
+    p.num_tiles = (int)tiles;
+    return true;
+}
+
+// Forward transform of one operand, or of two operands in one launch (pb may be null).
 template <int N, bool FREQ>
-static cudaError_t launch_r2c_n(FftParams p, cudaStream_t st) {
+static cudaError_t launch_r2c_n(FftParams pa, const FftParams* pb_in, cudaStream_t st) {
     using Cfg = FftCfg<N>;
     constexpr int G = Cfg::G;
     constexpr int LAYOUT = !FREQ ? LAYOUT_BARE : (Cfg::TMA ? LAYOUT_FREQ_TMA : LAYOUT_FREQ_DIRECT);
-    p.tiles_per_row = (p.C + G - 1) / G;
-    const long long tiles = (long long)p.R * p.tiles_per_row;
-    if (tiles <= 0 || tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
-    p.num_tiles = (int)tiles;
-    p.in_bytes = real_tile_bytes(G, p.h, p.w);
-    const size_t mid = MidGeom<N, G>::BYTES;
-    size_t smem = Cfg::ALIAS ? (mid > (size_t)p.in_bytes ? mid : (size_t)p.in_bytes)
-                             : mid + (size_t)p.in_bytes;
-    CUtensorMap tm;
-    memset(&tm, 0, sizeof(tm));
-    if (LAYOUT == LAYOUT_FREQ_TMA) {
-        smem += (size_t)2 * N * (N / 2 + 1) * G * sizeof(float);
-        if (!make_spec_map<N, G>(&tm, p.spec_out, p)) return cudaErrorInvalidValue;
+    FftParams pb{};
+    if (!fill_tiling<G>(pa)) return cudaErrorInvalidValue;
+    int in_bytes = real_tile_bytes(G, pa.h, pa.w);
+    if (pb_in) {
+        pb = *pb_in;
+        if (!fill_tiling<G>(pb)) return cudaErrorInvalidValue;
+        const int b = real_tile_bytes(G, pb.h, pb.w);
+        if (b > in_bytes) in_bytes = b;
     }
-    return launch_persistent(r2c_kernel<N, G, LAYOUT, Cfg::ALIAS, Cfg::MINB>, N * G, smem, tm, p, st);
+    pa.in_bytes = pb.in_bytes = in_bytes;
+    const size_t mid = MidGeom<N, G>::BYTES;
+    size_t smem = Cfg::ALIAS ? (mid > (size_t)in_bytes ? mid : (size_t)in_bytes) : mid + (size_t)in_bytes;
+    CUtensorMap tma, tmb;
+    memset(&tma, 0, sizeof(tma));
+    memset(&tmb, 0, sizeof(tmb));
+    constexpr bool SALIAS = Cfg::SALIAS && LAYOUT == LAYOUT_FREQ_TMA;
+    if (LAYOUT == LAYOUT_FREQ_TMA) {
+        const size_t stage = (size_t)2 * N * (N / 2 + 1) * G * sizeof(float);
+        if (SALIAS) smem = (size_t)in_bytes + (stage > mid ? stage : mid);
+        else smem += stage;
+        if (!make_spec_map<N, G>(&tma, pa.spec_out, pa)) return cudaErrorInvalidValue;
+        if (pb_in && !make_spec_map<N, G>(&tmb, pb.spec_out, pb)) return cudaErrorInvalidValue;
+    }
+    auto kern = r2c_kernel<N, G, LAYOUT, Cfg::ALIAS, SALIAS, Cfg::MINB>;
+    int grid = 0;
+    cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), N * G, smem,
+                                    (long long)pa.num_tiles + pb.num_tiles, &grid);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, N * G, smem, st>>>(tma, tmb, pa, pb);
+    return cudaGetLastError();
 }
 
 template <int N, bool FREQ>
@@ -608,10 +754,7 @@ static cudaError_t launch_c2r_n(FftParams p, cudaStream_t st) {
     using Cfg = FftCfg<N>;
     constexpr int G = Cfg::G;
     constexpr int LAYOUT = !FREQ ? LAYOUT_BARE : (Cfg::TMA ? LAYOUT_FREQ_TMA : LAYOUT_FREQ_DIRECT);
-    p.tiles_per_row = (p.C + G - 1) / G;
-    const long long tiles = (long long)p.R * p.tiles_per_row;
-    if (tiles <= 0 || tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
-    p.num_tiles = (int)tiles;
+    if (!fill_tiling<G>(p)) return cudaErrorInvalidValue;
     p.in_bytes = 0;
     size_t smem = MidGeom<N, G>::BYTES;
     CUtensorMap tm;
@@ -620,17 +763,22 @@ static cudaError_t launch_c2r_n(FftParams p, cudaStream_t st) {
         smem += (size_t)2 * N * (N / 2 + 1) * G * sizeof(float);
         if (!make_spec_map<N, G>(&tm, p.spec_in, p)) return cudaErrorInvalidValue;
     }
-    return launch_persistent(c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV>, N * G, smem, tm, p, st);
+    auto kern = c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV>;
+    int grid = 0;
+    cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), N * G, smem, p.num_tiles, &grid);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, N * G, smem, st>>>(tm, p);
+    return cudaGetLastError();
 }
 
 template <bool FREQ>
-static cudaError_t launch_r2c(int n, const FftParams& p, cudaStream_t st) {
+static cudaError_t launch_r2c(int n, const FftParams& p, const FftParams* second, cudaStream_t st) {
     switch (n) {
-        case 8:   return launch_r2c_n<8, FREQ>(p, st);
-        case 16:  return launch_r2c_n<16, FREQ>(p, st);
-        case 32:  return launch_r2c_n<32, FREQ>(p, st);
-        case 64:  return launch_r2c_n<64, FREQ>(p, st);
-        case 128: return launch_r2c_n<128, FREQ>(p, st);
+        case 8:   return launch_r2c_n<8, FREQ>(p, second, st);
+        case 16:  return launch_r2c_n<16, FREQ>(p, second, st);
+        case 32:  return launch_r2c_n<32, FREQ>(p, second, st);
+        case 64:  return launch_r2c_n<64, FREQ>(p, second, st);
+        case 128: return launch_r2c_n<128, FREQ>(p, second, st);
     }
     return cudaErrorInvalidValue;
 }
