@@ -132,16 +132,18 @@ int conv_plan_status(conv_plan_t* plan);
 int conv_plan_destroy(conv_plan_t* plan);
 
 /* Per-stage device timing for benchmarks.  enable != 0 makes every following
- * pass record CUDA events on its stream around each of its four kernels
- * (forward FFT of the first operand, forward FFT of the second, per-bin
- * contraction, inverse FFT -- the columns of the paper's Table 4 with the
- * transposes fused away).  Creates the events on first use (the only state the
+ * pass record CUDA events on its stream around its kernels -- the columns of the
+ * paper's Table 4 with the transposes fused away.  enable == 1 keeps the normal
+ * launch sequence (both forward FFTs in one kernel, per-bin contraction, inverse
+ * FFT); enable == 2 launches the two forward FFTs as separate kernels so that
+ * they can be timed apart.  Creates the events on first use (the only state the
  * plan owns on the device side). */
 int conv_plan_enable_stage_timing(conv_plan_t* plan, int enable);
 
-/* Waits for the last pass issued with timing enabled and writes the duration of
- * its four kernels in milliseconds to out_ms[0..3].  EINVAL if timing is off or
- * no pass has run. */
+/* Waits for the last pass issued with timing enabled and writes durations in
+ * milliseconds to out_ms[0..3]: forward FFT of the first operand (mode 1: of both
+ * operands, the one fused kernel), forward FFT of the second operand (mode 1:
+ * zero), contraction, inverse FFT.  EINVAL if timing is off or no pass has run. */
 int conv_plan_stage_times_ms(conv_plan_t* plan, float* out_ms);
 
 /* Bare batched 2-D real-to-complex transform (Supplement 8.2 definition,

@@ -205,13 +205,15 @@ def conv_plan_status(plan: Plan) -> int:
     return int(lib().conv_plan_status(plan.handle))
 
 
-def conv_plan_enable_stage_timing(plan: Plan, enable=True) -> None:
-    _check(lib().conv_plan_enable_stage_timing(plan.handle, int(bool(enable))),
+def conv_plan_enable_stage_timing(plan: Plan, enable=1) -> None:
+    """0 off; 1 time the normal launch sequence; 2 launch the two forward FFTs apart."""
+    _check(lib().conv_plan_enable_stage_timing(plan.handle, int(enable)),
            "conv_plan_enable_stage_timing")
 
 
 def conv_plan_stage_times_ms(plan: Plan):
-    """Milliseconds of the last timed pass's four kernels: fft A, fft B, contraction, ifft."""
+    """Milliseconds of the last timed pass: forward FFT A (mode 1: A and B fused), forward
+    FFT B (mode 1: 0), contraction, inverse FFT."""
     buf = (ctypes.c_float * 4)()
     _check(lib().conv_plan_stage_times_ms(plan.handle, ctypes.cast(buf, ctypes.c_void_p)),
            "conv_plan_stage_times_ms")
