@@ -66,8 +66,13 @@ int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, int w, int kh,
  * workspace size: query it again afterwards. */
 int conv_plan_set_math(conv_plan_t* plan, int math);
 
-/* Math mode the plan will actually run (FFTCONV_MATH_FP32 or _TF32) once AUTO is resolved. */
+/* Math mode the plan actually runs once AUTO is resolved.  The three passes
+ * contract over different indices (f, f', S), so AUTO resolves per pass:
+ * conv_plan_pass_math returns FFTCONV_MATH_FP32 or _TF32 for pass 0 (fprop),
+ * 1 (bprop) or 2 (accGrad); conv_plan_effective_math returns _TF32 only if all
+ * three passes run on the tensor cores, else _FP32. */
 int conv_plan_effective_math(const conv_plan_t* plan);
+int conv_plan_pass_math(const conv_plan_t* plan, int pass);
 
 /* Bytes of device scratch the three passes need: the frequency-domain copies of
  * the two operands and of the result (Section 6 lists the same buffers), in the

@@ -17,7 +17,8 @@ EINVAL, EUNSUPPORTED, EWORKSPACE, ECUDA, EDEVICE_TIMEOUT = -1, -2, -3, -4, -5
 MATH_AUTO, MATH_FP32, MATH_TF32 = 0, 1, 2
 
 EXPORTS = (
-    "conv_plan", "conv_plan_set_math", "conv_plan_effective_math", "conv_plan_workspace_bytes",
+    "conv_plan", "conv_plan_set_math", "conv_plan_effective_math", "conv_plan_pass_math",
+    "conv_plan_workspace_bytes",
     "conv_plan_set_workspace", "conv_fprop", "conv_fprop_noalloc", "conv_bprop", "conv_accgrad", "conv_plan_status",
     "conv_plan_destroy", "conv_plan_enable_stage_timing", "conv_plan_stage_times_ms", "fft2d_r2c", "fft2d_c2r", "fftconv_bin_contract",
     "fftconv_status_string", "fftconv_launch_count",
@@ -45,6 +46,7 @@ def lib():
         L.conv_plan.argtypes = [ctypes.POINTER(p)] + [i] * 8
         L.conv_plan_set_math.argtypes = [p, i]
         L.conv_plan_effective_math.argtypes = [p]
+        L.conv_plan_pass_math.argtypes = [p, i]
         L.conv_plan_workspace_bytes.argtypes = [p]
         L.conv_plan_workspace_bytes.restype = z
         L.conv_plan_set_workspace.argtypes = [p, p, z]
@@ -139,6 +141,14 @@ def conv_plan_set_math(plan: Plan, math: int) -> None:
 
 def conv_plan_effective_math(plan: Plan) -> int:
     return int(lib().conv_plan_effective_math(plan.handle))
+
+
+def conv_plan_pass_math(plan: Plan, which: int) -> int:
+    """Math mode of pass 0 (fprop), 1 (bprop) or 2 (accGrad) once AUTO is resolved."""
+    r = int(lib().conv_plan_pass_math(plan.handle, int(which)))
+    if r < 0:
+        raise FftConvError(r, "conv_plan_pass_math")
+    return r
 
 
 def conv_plan_workspace_bytes(plan: Plan) -> int:

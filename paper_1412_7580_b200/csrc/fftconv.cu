@@ -220,6 +220,11 @@ FFTCONV_API int conv_plan_effective_math(const conv_plan_t* plan) {
     return FFTCONV_MATH_TF32;
 }
 
+FFTCONV_API int conv_plan_pass_math(const conv_plan_t* plan, int pass) {
+    if (!plan || pass < 0 || pass > 2) return FFTCONV_EINVAL;
+    return resolve_math(*plan, describe(*plan, pass));
+}
+
 FFTCONV_API size_t conv_plan_workspace_bytes(const conv_plan_t* plan) {
     if (!plan) return 0;
     size_t m = 0;

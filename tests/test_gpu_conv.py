@@ -37,7 +37,7 @@ def run_gpu(shape, x, w, dy, math, accumulate_init=None):
     fc.conv_accgrad(p, dyd, xd, dw)
     torch.cuda.synchronize()
     assert fc.conv_plan_status(p) == 0
-    eff = fc.conv_plan_effective_math(p)
+    eff = [fc.conv_plan_pass_math(p, k) for k in range(3)]     # AUTO resolves per pass
     res = (y.cpu().numpy().astype(np.float64), dx.cpu().numpy().astype(np.float64),
            dw.cpu().numpy().astype(np.float64), eff)
     fc.conv_plan_destroy(p)
@@ -72,12 +72,11 @@ def test_small_shapes_full_tensors(dims, math):
     s = wl.ConvShape("case", *dims, cfg=7, point=sum(dims))
     x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
     y, dx, dw, eff = run_gpu(s, x, w, dy, math)
-    tol = TOL[eff]
     for got in (y, dx, dw):
         assert np.all(np.isfinite(got))
-    assert relerr(y, oracle.fprop(x, w)) <= tol
-    assert relerr(dx, oracle.bprop(dy, w, s.h, s.w)) <= tol
-    assert relerr(dw, oracle.accgrad(dy, x, s.kh, s.kw)) <= tol
+    assert relerr(y, oracle.fprop(x, w)) <= TOL[eff[0]]
+    assert relerr(dx, oracle.bprop(dy, w, s.h, s.w)) <= TOL[eff[1]]
+    assert relerr(dw, oracle.accgrad(dy, x, s.kh, s.kw)) <= TOL[eff[2]]
 
 
 def test_accgrad_accumulates():
@@ -107,19 +106,19 @@ def test_benchmark_layers_sampled(cfg, math):
     s = wl.CONFIGS[cfg]
     x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
     y, dx, dw, eff = run_gpu(s, x, w, dy, math)
-    tol = TOL[eff]
+    tol = max(TOL[e] for e in eff)
     for got in (y, dx, dw):
         assert np.all(np.isfinite(got))
     # normalisation: max-abs of the sampled oracle values (close to the tensor's)
     cy = wl.sample_coords(y.shape, 4000, seed=cfg)
     ry = oracle.fprop_at(x, w, cy)
-    assert relerr(y[cy[:, 0], cy[:, 1], cy[:, 2], cy[:, 3]], ry) <= tol
+    assert relerr(y[cy[:, 0], cy[:, 1], cy[:, 2], cy[:, 3]], ry) <= TOL[eff[0]]
     cx = wl.sample_coords(dx.shape, 4000, seed=cfg + 10)
     rx = oracle.bprop_at(dy, w, s.h, s.w, cx)
-    assert relerr(dx[cx[:, 0], cx[:, 1], cx[:, 2], cx[:, 3]], rx) <= tol
+    assert relerr(dx[cx[:, 0], cx[:, 1], cx[:, 2], cx[:, 3]], rx) <= TOL[eff[1]]
     cw = wl.sample_coords(dw.shape, 600, seed=cfg + 20)
     rw = oracle.accgrad_at(dy, x, s.kh, s.kw, cw)
-    assert relerr(dw[cw[:, 0], cw[:, 1], cw[:, 2], cw[:, 3]], rw) <= tol
+    assert relerr(dw[cw[:, 0], cw[:, 1], cw[:, 2], cw[:, 3]], rw) <= TOL[eff[2]]
     # adjoint identity on the full GPU tensors: <y,dy> = <x,dx> = <w,dw>
     a = float(np.sum(y * dy)); b = float(np.sum(dx * x)); c = float(np.sum(dw * w))
     scale = np.sqrt(float(np.sum(y * y)) * float(np.sum(dy.astype(np.float64) ** 2)))
@@ -136,12 +135,11 @@ def test_sweep_subset():
     for s in pts:
         x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
         y, dx, dw, eff = run_gpu(s, x, w, dy, 0)
-        tol = TOL[eff]
         cy = wl.sample_coords(y.shape, 300, seed=s.point)
-        assert relerr(y[cy[:, 0], cy[:, 1], cy[:, 2], cy[:, 3]], oracle.fprop_at(x, w, cy)) <= tol, s
+        assert relerr(y[cy[:, 0], cy[:, 1], cy[:, 2], cy[:, 3]], oracle.fprop_at(x, w, cy)) <= TOL[eff[0]], s
         cx = wl.sample_coords(dx.shape, 300, seed=s.point + 1)
         assert relerr(dx[cx[:, 0], cx[:, 1], cx[:, 2], cx[:, 3]],
-                      oracle.bprop_at(dy, w, s.h, s.w, cx)) <= tol, s
+                      oracle.bprop_at(dy, w, s.h, s.w, cx)) <= TOL[eff[1]], s
         cw = wl.sample_coords(dw.shape, 60, seed=s.point + 2)
         assert relerr(dw[cw[:, 0], cw[:, 1], cw[:, 2], cw[:, 3]],
-                      oracle.accgrad_at(dy, x, s.kh, s.kw, cw)) <= tol, s
+                      oracle.accgrad_at(dy, x, s.kh, s.kw, cw)) <= TOL[eff[2]], s
