@@ -220,17 +220,19 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
     const int kyp = u / G, gB = u - kyp * G;
     const int q4 = tid / (T / 4), u4 = tid - q4 * (T / 4);      // step 2, narrow planes: quarter
     // operand-dependent state, set by select()
-    int h, w, hw, opC;
-    int gA, cA, g4, c4;                                         // step 2: (plane, column)
-    bool split4;                                                // narrow planes: 4 threads per column
+    int h = 1, w = 1, hw = 1, opC = 1, tpr = 1, step_rows = 0, step_cols = 0;
+    int gA = 0, cA = 0, g4 = 0, c4 = 0;                         // step 2: (plane, column)
+    bool split4 = false;                                        // narrow planes: 4 threads per column
     auto select = [&](bool second) {
         h = second ? p1.h : p0.h;
         w = second ? p1.w : p0.w;
         opC = second ? p1.C : p0.C;
+        tpr = second ? p1.tiles_per_row : p0.tiles_per_row;
         hw = h * w;
         gA = tid / w; cA = tid - gA * w;
         split4 = (4 * G * w <= T);
         g4 = u4 / w; c4 = u4 - g4 * w;
+        step_rows = gridDim.x / tpr; step_cols = gridDim.x - step_rows * tpr;
     };
     // tile index -> (operand, row, tile in row)
     auto locate = [&](int tile, bool& second, int& row, int& tcol) {
@@ -284,6 +286,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
     if ((int)blockIdx.x < total_tiles) {
         locate(blockIdx.x, second_n, row_n, tcol_n);
         pending = stage(second_n, row_n, tcol_n);
+        select(second_n);
     }
     __syncthreads();           // plain-load parts of the first tile are visible to everyone
 
@@ -291,14 +294,21 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
     long long tl_last = clock64();
 #endif
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        if (second_n != second) select(second_n);       // divisions only when the operand changes
         second = second_n; row = row_n; tcol = tcol_n;
-        select(second);
         const FftParams& p = second ? p1 : p0;
         const CUtensorMap* tmS = second ? &tmS1 : &tmS0;
         const int c0 = tcol * G;
         const int gcount = min(G, opC - c0);
         const int next = tile + gridDim.x;
-        if (next < total_tiles) locate(next, second_n, row_n, tcol_n);
+        if (next < total_tiles) {
+            if (!second && next >= p0.num_tiles) {
+                locate(next, second_n, row_n, tcol_n);  // crossing into the second operand
+            } else {
+                row_n = row + step_rows; tcol_n = tcol + step_cols;
+                if (tcol_n >= tpr) { tcol_n -= tpr; ++row_n; }
+            }
+        }
 
         FC_TICK(0);
         if (pending) {
@@ -666,7 +676,7 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
 template <int N> struct FftCfg;   // planes per CTA, buffer aliasing, min CTAs per SM, TMA staging
 template <> struct FftCfg<8>   { static constexpr int G = 32; static constexpr bool ALIAS = false, SALIAS = true;  static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
 template <> struct FftCfg<16>  { static constexpr int G = 16; static constexpr bool ALIAS = false, SALIAS = true;  static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
-template <> struct FftCfg<32>  { static constexpr int G = 8;  static constexpr bool ALIAS = false, SALIAS = true;  static constexpr int MINB = 3, MINB_INV = 3; static constexpr bool TMA = true; };
+template <> struct FftCfg<32>  { static constexpr int G = 8;  static constexpr bool ALIAS = false, SALIAS = true;  static constexpr int MINB = 2, MINB_INV = 3; static constexpr bool TMA = true; };
 template <> struct FftCfg<64>  { static constexpr int G = 4;  static constexpr bool ALIAS = false, SALIAS = false; static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = true; };
 template <> struct FftCfg<128> { static constexpr int G = 2;  static constexpr bool ALIAS = true,  SALIAS = false; static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = false; };
 
