@@ -221,7 +221,6 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
     const int q4 = tid / (T / 4), u4 = tid - q4 * (T / 4);      // step 2, narrow planes: quarter
     // operand-dependent state, set by select()
     int h = 1, w = 1, hw = 1, opC = 1, tpr = 1, step_rows = 0, step_cols = 0;
-    int gA = 0, cA = 0, g4 = 0, c4 = 0;                         // step 2: (plane, column)
     bool split4 = false;                                        // narrow planes: 4 threads per column
     auto select = [&](bool second) {
         h = second ? p1.h : p0.h;
@@ -229,11 +228,14 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
         opC = second ? p1.C : p0.C;
         tpr = second ? p1.tiles_per_row : p0.tiles_per_row;
         hw = h * w;
-        gA = tid / w; cA = tid - gA * w;
-        split4 = (4 * G * w <= T);
-        g4 = u4 / w; c4 = u4 - g4 * w;
+        split4 = (4 * w <= N);
         step_rows = gridDim.x / tpr; step_cols = gridDim.x - step_rows * tpr;
     };
+    // step 2 roles: N lanes per plane (a warp never straddles two planes, so neither its
+    // reads of the real tile nor its writes to the scratch collide on a bank); narrow planes
+    // use N/4 lanes per plane and quarter
+    const int gA = tid / N, cA = tid % N;
+    const int g4 = u4 / (N / 4), c4 = u4 % (N / 4);
     // tile index -> (operand, row, tile in row)
     auto locate = [&](int tile, bool& second, int& row, int& tcol) {
         second = tile >= p0.num_tiles;
@@ -327,7 +329,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             float br[L], bi[L];
             bool act;
             if (!split4) {
-                act = (gA < gcount);                    // gA < G follows from tid < G*w
+                act = (gA < gcount) && (cA < w);
                 if (act) {
                     float v[N];
                     const float* src = sIn + gA * hw + cA;
@@ -338,7 +340,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
                     rfft<N>(v, Xr, Xi);
                 }
             } else {
-                act = (u4 < G * w) && (g4 < gcount);
+                act = (c4 < w) && (g4 < gcount);
                 if (act) {
                     const float* src = sIn + g4 * hw + c4;
                     auto quarter = [&](auto Q) {
@@ -528,7 +530,7 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
 
     const int tid = threadIdx.x;
     const int hc = p.h, wc = p.w, hw = hc * wc;
-    const int gA = tid / wc, cA = tid - gA * wc;                // step 2: (plane, column)
+    const int gA = tid / N, cA = tid % N;                       // step 2: (plane, column), N lanes per plane
     const int q = tid / HALF, u = tid - q * HALF;               // step 1: (half, row ky, plane)
     const int kyp = u / G, gB = u - kyp * G;
     const bool packed = (kyp == 0);
@@ -641,7 +643,7 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
 
         // 2. column transforms: thread = (plane gA, column cA), cA < wc; results go straight
         //    to global memory (lanes run along the row of the plane: contiguous segments)
-        if (gA < gcount) {
+        if (gA < gcount && cA < wc) {
             float v[N];
             {
                 float Xr[NC], Xi[NC];
