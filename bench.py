@@ -34,9 +34,9 @@ FP32_FFMA_TFLOPS_NOMINAL = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x lanes x 2 fl
 # DRAM bytes (read + write) of one launch from the ncu captures summarised under profiles/,
 # keyed by (workload, kernel, pass); None where no capture exists.
 NCU_TRAFFIC = {
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "bprop"): 295.8e6,
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "accgrad"): 290.0e6,
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "fprop"): 160.9e6,
+    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "bprop"): 291.9e6,
+    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "accgrad"): 287.2e6,
+    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "fprop"): 156.6e6,
 }
 
 
