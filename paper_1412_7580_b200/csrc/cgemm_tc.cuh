@@ -390,12 +390,14 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 template <bool TA, bool TB>
 static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStream_t st, int sm_count) {
     auto kern = cgemm_tc_kernel<TA, TB>;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static unsigned long long attr_set_devices = 0;     // one bit per device ordinal
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    if (dev >= 64 || !((attr_set_devices >> dev) & 1ull)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)TC_SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        attr_set = true;
+        if (dev < 64) attr_set_devices |= 1ull << dev;
     }
     CUtensorMap tmA, tmB, tmC;
     // k-contiguous: rows = M (or N), cols = K, box 32 k x 128 rows;

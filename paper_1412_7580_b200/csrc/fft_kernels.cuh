@@ -43,6 +43,8 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "fft_core.cuh"
 #include "tma_util.cuh"
 
@@ -693,15 +695,44 @@ static inline int fft_sm_count() {
     return sms;
 }
 
+// Grid of a persistent kernel: one CTA per resident slot.  The attribute call and the
+// occupancy query cost microseconds of host time each, so their result is remembered per
+// (kernel, shared-memory size).
 static cudaError_t persistent_grid(const void* kern, int threads, size_t smem, long long tiles,
                                    int* grid) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+    struct Entry { const void* kern; size_t smem; int dev; int per_sm; };
+    struct Limit { const void* kern; int dev; size_t max_smem; };
+    static Entry cache[128];
+    static Limit limits[64];
+    static int cached = 0, nlimits = 0;
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    // the opt-in shared-memory limit of a kernel is only ever raised
+    Limit* lim = nullptr;
+    for (int i = 0; i < nlimits; ++i)
+        if (limits[i].kern == kern && limits[i].dev == dev) lim = &limits[i];
+    if (!lim || lim->max_smem < smem) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        if (lim) lim->max_smem = smem;
+        else if (nlimits < 64) limits[nlimits++] = Limit{kern, dev, smem};
+    }
     int per_sm = 0;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
-    if (e != cudaSuccess) return e;
+    for (int i = 0; i < cached; ++i)
+        if (cache[i].kern == kern && cache[i].smem == smem && cache[i].dev == dev) {
+            per_sm = cache[i].per_sm;
+            break;
+        }
+    if (per_sm == 0) {
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, threads, smem);
+        if (e != cudaSuccess) return e;
+        if (per_sm < 1) return cudaErrorInvalidConfiguration;
+        if (cached < 128) cache[cached++] = Entry{kern, smem, dev, per_sm};
+    }
     const int sms = fft_sm_count();
-    if (per_sm < 1 || sms < 1) return cudaErrorInvalidConfiguration;
+    if (sms < 1) return cudaErrorInvalidConfiguration;
     const long long slots = (long long)per_sm * sms;
     *grid = (int)(tiles < slots ? tiles : slots);
     return cudaSuccess;
