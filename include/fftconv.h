@@ -128,6 +128,23 @@ int conv_bprop(conv_plan_t* plan, const float* dy, const float* w, float* dx, vo
 int conv_accgrad(conv_plan_t* plan, const float* dy, const float* x, float* dw, int accumulate,
                  void* cuda_stream);
 
+/* Spectrum reuse across the passes of one training step (the paper's Section 6
+ * notes that the forward transforms could be shared between passes, saving a
+ * third of them, and passes on it for memory reasons).  With enable != 0 the
+ * workspace holds one region per tensor family (x, w, dy) plus one for the
+ * result spectrum -- query conv_plan_workspace_bytes again and lend a workspace
+ * of that size -- and the spectra survive a pass: conv_fprop always transforms x
+ * and w afresh; conv_bprop transforms dy and takes w's spectrum from the
+ * preceding conv_fprop if it is given the same w pointer; conv_accgrad takes
+ * dy's and x's spectra from the preceding passes if given the same pointers.
+ * A tensor passed under a pointer whose spectrum is cached must not have been
+ * modified since that spectrum was computed, and the passes must be ordered on
+ * one stream (or synchronised by the caller); otherwise call
+ * conv_plan_invalidate_spectra first.  Changing the setting or the workspace
+ * invalidates everything.  Results are identical to the non-reusing passes. */
+int conv_plan_set_spectrum_reuse(conv_plan_t* plan, int enable);
+int conv_plan_invalidate_spectra(conv_plan_t* plan);
+
 /* Reads the plan's device status word (synchronises the device).  FFTCONV_OK,
  * or FFTCONV_EDEVICE_TIMEOUT if a bounded wait inside a kernel gave up since
  * the last call (the word is then cleared), or ECUDA. */

@@ -19,7 +19,8 @@ MATH_AUTO, MATH_FP32, MATH_TF32 = 0, 1, 2
 EXPORTS = (
     "conv_plan", "conv_plan_set_math", "conv_plan_effective_math", "conv_plan_pass_math",
     "conv_plan_workspace_bytes",
-    "conv_plan_set_workspace", "conv_fprop", "conv_fprop_noalloc", "conv_bprop", "conv_accgrad", "conv_plan_status",
+    "conv_plan_set_workspace", "conv_plan_set_spectrum_reuse", "conv_plan_invalidate_spectra",
+    "conv_fprop", "conv_fprop_noalloc", "conv_bprop", "conv_accgrad", "conv_plan_status",
     "conv_plan_destroy", "conv_plan_enable_stage_timing", "conv_plan_stage_times_ms", "fft2d_r2c", "fft2d_c2r", "fftconv_bin_contract",
     "fftconv_status_string", "fftconv_launch_count",
 )
@@ -50,6 +51,8 @@ def lib():
         L.conv_plan_workspace_bytes.argtypes = [p]
         L.conv_plan_workspace_bytes.restype = z
         L.conv_plan_set_workspace.argtypes = [p, p, z]
+        L.conv_plan_set_spectrum_reuse.argtypes = [p, i]
+        L.conv_plan_invalidate_spectra.argtypes = [p]
         L.conv_fprop.argtypes = [p, p, p, p, p]
         L.conv_fprop_noalloc.argtypes = [p, p, p, p, p]
         L.conv_bprop.argtypes = [p, p, p, p, p]
@@ -161,6 +164,17 @@ def conv_plan_set_workspace(plan: Plan, workspace) -> None:
     _check(lib().conv_plan_set_workspace(plan.handle, ctypes.c_void_p(workspace.data_ptr()),
                                          nbytes), "conv_plan_set_workspace")
     plan.workspace = workspace
+
+
+def conv_plan_set_spectrum_reuse(plan: Plan, enable=True) -> None:
+    """Keep the forward spectra between fprop / bprop / accGrad of one step (changes the
+    workspace size: size and lend the workspace after this call)."""
+    _check(lib().conv_plan_set_spectrum_reuse(plan.handle, int(bool(enable))),
+           "conv_plan_set_spectrum_reuse")
+
+
+def conv_plan_invalidate_spectra(plan: Plan) -> None:
+    _check(lib().conv_plan_invalidate_spectra(plan.handle), "conv_plan_invalidate_spectra")
 
 
 def conv_plan_alloc_workspace(plan: Plan, device="cuda"):

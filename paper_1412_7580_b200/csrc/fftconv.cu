@@ -38,6 +38,7 @@ struct SpecDesc {
 struct OperandDesc {
     SpecDesc spec;
     int h, w;               // plane size (forward) or crop window (inverse)
+    int kind;               // which tensor family: 0 = x / dx, 1 = w / dw, 2 = y / dy
 };
 
 struct PassDesc {
@@ -56,6 +57,8 @@ struct conv_plan_s {
     int math;          // requested fftconv_math
     void* ws;
     size_t ws_bytes;
+    int reuse;              // keep the forward spectra between the passes of a training step
+    const float* cached[3]; // reuse: tensor whose spectrum sits in region 0 (x), 1 (w), 2 (dy)
     int timing;             // record events around the four kernels of a pass
     bool timed;             // a timed pass has been issued
     cudaEvent_t ev[5];
@@ -75,9 +78,9 @@ namespace {
 PassDesc describe(const conv_plan_s& p, int pass) {
     PassDesc d{};
     auto spec = [](int R, int C) { return SpecDesc{R, C, round4(C)}; };
-    const OperandDesc X = {spec(p.S, p.f), p.h, p.w};
-    const OperandDesc W = {spec(p.fp, p.f), p.kh, p.kw};
-    const OperandDesc Y = {spec(p.S, p.fp), p.oh, p.ow};
+    const OperandDesc X = {spec(p.S, p.f), p.h, p.w, 0};
+    const OperandDesc W = {spec(p.fp, p.f), p.kh, p.kw, 1};
+    const OperandDesc Y = {spec(p.S, p.fp), p.oh, p.ow, 2};
     switch (pass) {
         case PASS_FPROP:
             d.a = X; d.b = W; d.c = Y;
@@ -125,6 +128,28 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
                                             align_up(d.a.spec.bytes(plan->bins), kAlign));
     float* specC = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(specB) +
                                             align_up(d.b.spec.bytes(plan->bins), kAlign));
+    // Which forward transforms this pass has to run.  Without reuse: both.  With reuse the
+    // spectra live in fixed per-tensor regions and survive the pass: fprop always refreshes
+    // x and w (new data every step), bprop refreshes dy and takes w's spectrum from fprop,
+    // accGrad takes both from the earlier passes -- whenever the same device pointer is
+    // passed again; otherwise the spectrum is recomputed.
+    bool need_a = true, need_b = true;
+    if (plan->reuse) {
+        const PassDesc f = describe(*plan, PASS_FPROP);
+        unsigned char* r0 = base + kHeaderBytes;
+        unsigned char* r1 = r0 + align_up(f.a.spec.bytes(plan->bins), kAlign);
+        unsigned char* r2 = r1 + align_up(f.b.spec.bytes(plan->bins), kAlign);
+        unsigned char* r3 = r2 + align_up(f.c.spec.bytes(plan->bins), kAlign);
+        unsigned char* region[3] = {r0, r1, r2};
+        specA = reinterpret_cast<float*>(region[d.a.kind]);
+        specB = reinterpret_cast<float*>(region[d.b.kind]);
+        specC = reinterpret_cast<float*>(r3);
+        const bool fresh_a = (pass != PASS_ACCGRAD), fresh_b = (pass == PASS_FPROP);
+        need_a = fresh_a || plan->cached[d.a.kind] != a_in;
+        need_b = fresh_b || plan->cached[d.b.kind] != b_in;
+        plan->cached[d.a.kind] = a_in;
+        plan->cached[d.b.kind] = b_in;
+    }
 
     auto operand = [&](const OperandDesc& o, const float* in, float* spec) {
         fc::FftParams fp{};
@@ -137,7 +162,15 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     auto mark = [&](int i) { if (timing) cudaEventRecord(plan->ev[i], st); };
     mark(0);
     const fc::FftParams fa = operand(d.a, a_in, specA), fb = operand(d.b, b_in, specB);
-    if (!timing || plan->timing == 1) {
+    if (!need_a || !need_b) {
+        // spectrum reuse: at most one operand left to transform
+        if (need_a || need_b) {
+            g_launches.fetch_add(1, std::memory_order_relaxed);
+            if (fc::launch_r2c<true>(plan->n, need_a ? fa : fb, nullptr, st) != cudaSuccess)
+                return FFTCONV_ECUDA;
+        }
+        mark(1);
+    } else if (!timing || plan->timing == 1) {
         // both forward transforms in one launch: one ramp-up, one tail
         g_launches.fetch_add(1, std::memory_order_relaxed);
         if (fc::launch_r2c<true>(plan->n, fa, &fb, st) != cudaSuccess) return FFTCONV_ECUDA;
@@ -200,6 +233,7 @@ FFTCONV_API int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, in
     p->math = FFTCONV_MATH_AUTO;
     p->ws = nullptr; p->ws_bytes = 0;
     p->timing = 0; p->timed = false; p->ev_made = false;
+    p->reuse = 0; p->cached[0] = p->cached[1] = p->cached[2] = nullptr;
     *out = p;
     return FFTCONV_OK;
 }
@@ -227,6 +261,15 @@ FFTCONV_API int conv_plan_pass_math(const conv_plan_t* plan, int pass) {
 
 FFTCONV_API size_t conv_plan_workspace_bytes(const conv_plan_t* plan) {
     if (!plan) return 0;
+    if (plan->reuse) {
+        // one region per tensor family plus one for the result spectrum of the running pass
+        const PassDesc d = describe(*plan, PASS_FPROP);      // a = x, b = w, c = y
+        const size_t bx = align_up(d.a.spec.bytes(plan->bins), kAlign),
+                     bw = align_up(d.b.spec.bytes(plan->bins), kAlign),
+                     by = align_up(d.c.spec.bytes(plan->bins), kAlign);
+        const size_t br = bx > bw ? (bx > by ? bx : by) : (bw > by ? bw : by);
+        return kHeaderBytes + bx + bw + by + br;
+    }
     size_t m = 0;
     for (int pass = 0; pass < 3; ++pass) {
         size_t b = pass_bytes(*plan, pass);
@@ -243,6 +286,20 @@ FFTCONV_API int conv_plan_set_workspace(conv_plan_t* plan, void* dev_ptr, size_t
     if (cudaMemset(dev_ptr, 0, kHeaderBytes) != cudaSuccess) return FFTCONV_ECUDA;
     plan->ws = dev_ptr;
     plan->ws_bytes = bytes;
+    plan->cached[0] = plan->cached[1] = plan->cached[2] = nullptr;
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_plan_set_spectrum_reuse(conv_plan_t* plan, int enable) {
+    if (!plan) return FFTCONV_EINVAL;
+    plan->reuse = enable ? 1 : 0;
+    plan->cached[0] = plan->cached[1] = plan->cached[2] = nullptr;
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_plan_invalidate_spectra(conv_plan_t* plan) {
+    if (!plan) return FFTCONV_EINVAL;
+    plan->cached[0] = plan->cached[1] = plan->cached[2] = nullptr;
     return FFTCONV_OK;
 }
 
@@ -279,7 +336,11 @@ void* noalloc_scratch_address() {
 FFTCONV_API int conv_fprop_noalloc(conv_plan_t* plan, const float* x, const float* w, float* y,
                                    void* cuda_stream) {
     if (!plan || !x || !w || !y) return FFTCONV_EINVAL;
-    if (conv_plan_workspace_bytes(plan) > (size_t)FFTCONV_NOALLOC_BYTES) return FFTCONV_EWORKSPACE;
+    {
+        conv_plan_s sized = *plan;      // the size of the ordinary (no-reuse) workspace layout
+        sized.reuse = 0;
+        if (conv_plan_workspace_bytes(&sized) > (size_t)FFTCONV_NOALLOC_BYTES) return FFTCONV_EWORKSPACE;
+    }
     void* scratch = noalloc_scratch_address();
     if (!scratch) return FFTCONV_ECUDA;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
@@ -289,6 +350,7 @@ FFTCONV_API int conv_fprop_noalloc(conv_plan_t* plan, const float* x, const floa
     conv_plan_s local = *plan;          // same shape and math mode, library-owned scratch
     local.ws = scratch;
     local.ws_bytes = FFTCONV_NOALLOC_BYTES;
+    local.reuse = 0;
     local.timing = 0;
     local.timed = false;
     local.ev_made = false;
