@@ -679,8 +679,8 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
 // ---------------------------------------------------------------------------
 template <int N> struct FftCfg;   // planes per CTA, buffer aliasing, min CTAs per SM, TMA staging
 template <> struct FftCfg<8>   { static constexpr int G = 32; static constexpr bool ALIAS = false, SALIAS = true;  static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
-template <> struct FftCfg<16>  { static constexpr int G = 16; static constexpr bool ALIAS = false, SALIAS = true;  static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
-template <> struct FftCfg<32>  { static constexpr int G = 8;  static constexpr bool ALIAS = false, SALIAS = true;  static constexpr int MINB = 2, MINB_INV = 3; static constexpr bool TMA = true; };
+template <> struct FftCfg<16>  { static constexpr int G = 16; static constexpr bool ALIAS = false, SALIAS = false;  static constexpr int MINB = 4, MINB_INV = 4; static constexpr bool TMA = true; };
+template <> struct FftCfg<32>  { static constexpr int G = 8;  static constexpr bool ALIAS = false, SALIAS = false;  static constexpr int MINB = 2, MINB_INV = 3; static constexpr bool TMA = true; };
 template <> struct FftCfg<64>  { static constexpr int G = 4;  static constexpr bool ALIAS = false, SALIAS = false; static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = true; };
 template <> struct FftCfg<128> { static constexpr int G = 2;  static constexpr bool ALIAS = true,  SALIAS = false; static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = false; };
 
