@@ -76,7 +76,7 @@ struct FftParams {
 template <int N, int G>
 struct MidGeom {
     static constexpr int PW = N + 1;
-    static constexpr int NEED = (N / 2 + 1) * PW;
+    static constexpr int NEED = (N / 2 + 1) * PW;   // the forward kernel uses N/2 rows of it
     static constexpr int UNIT = 16 / (G < 16 ? G : 16);
     static constexpr int MUL = ((NEED + UNIT - 1) / UNIT) | 1;
     static constexpr int P = MUL * UNIT;
@@ -179,6 +179,31 @@ __device__ __forceinline__ void load_split(Load&& load, float (&ar)[N / 2], floa
     });
 }
 
+// The same step when only the first N/2 inputs can be non-zero (zero-padded rows of a
+// narrow plane): the butterflies degenerate to a copy (q = 0) or one twiddle (q = 1).
+// `live` is the number of inputs that exist; the rest read as zero.
+template <int N, bool INV, int Q, class Load>
+__device__ __forceinline__ void load_split_narrow(Load&& load, int live, float (&ar)[N / 2],
+                                                  float (&ai)[N / 2]) {
+    constexpr int M = N / 2;
+    static_for<M>([&](auto J) {
+        constexpr int j = decltype(J)::value;
+        float2 lo = make_float2(0.0f, 0.0f);
+        if (j < live) lo = load(J);
+        if constexpr (Q == 0 || j == 0) {
+            ar[j] = lo.x; ai[j] = lo.y;
+        } else if constexpr (4 * j == N) {
+            if constexpr (!INV) { ar[j] = lo.y; ai[j] = -lo.x; }
+            else                { ar[j] = -lo.y; ai[j] = lo.x; }
+        } else {
+            constexpr float c = Tw<N, j>::c;
+            constexpr float sn = INV ? -Tw<N, j>::s : Tw<N, j>::s;
+            ar[j] = fc_fma(sn, lo.y, c * lo.x);
+            ai[j] = fc_fma(-sn, lo.x, c * lo.y);
+        }
+    });
+}
+
 #ifdef FC_EXP_TIMELINE
 __device__ long long fc_timeline[16];
 #define FC_TICK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { long long t_ = clock64(); fc_timeline[i] += t_ - tl_last; tl_last = t_; } } while (0)
@@ -224,6 +249,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
     // operand-dependent state, set by select()
     int h = 1, w = 1, hw = 1, opC = 1, tpr = 1, step_rows = 0, step_cols = 0;
     bool split4 = false;                                        // narrow planes: 4 threads per column
+    bool narrow = false;                                        // at most half the columns are live
     auto select = [&](bool second) {
         h = second ? p1.h : p0.h;
         w = second ? p1.w : p0.w;
@@ -231,6 +257,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
         tpr = second ? p1.tiles_per_row : p0.tiles_per_row;
         hw = h * w;
         split4 = (4 * w <= N);
+        narrow = (2 * w <= N);
         step_rows = gridDim.x / tpr; step_cols = gridDim.x - step_rows * tpr;
     };
     // step 2 roles: N lanes per plane (a warp never straddles two planes, so neither its
@@ -335,10 +362,27 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
                 if (act) {
                     float v[N];
                     const float* src = sIn + gA * hw + cA;
-                    static_for<N>([&](auto Rr) {
-                        constexpr int r = decltype(Rr)::value;
-                        v[r] = (r < h) ? src[r * w] : 0.0f;
-                    });
+                    // Zero-padding below the plane.  Rows r < N/2 exist whenever h > N/2 (the
+                    // usual case: N is the next power of two), so they are plain loads; the
+                    // others are loaded unconditionally (clamped) and zeroed by a select --
+                    // a branch per element would serialise the shared-memory loads.
+                    if (h > M) {
+                        static_for<N>([&](auto Rr) {
+                            constexpr int r = decltype(Rr)::value;
+                            if constexpr (r < M + 1) {
+                                v[r] = src[r * w];
+                            } else {
+                                const float t = src[min(r, h - 1) * w];
+                                v[r] = (r < h) ? t : 0.0f;
+                            }
+                        });
+                    } else {
+                        static_for<N>([&](auto Rr) {
+                            constexpr int r = decltype(Rr)::value;
+                            if constexpr (r < M) v[r] = (r < h) ? src[r * w] : 0.0f;
+                            else v[r] = 0.0f;
+                        });
+                    }
                     rfft<N>(v, Xr, Xi);
                 }
             } else {
@@ -380,20 +424,33 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             __syncthreads();   // tile consumed (and the previous tile's step 3 is done with sMid)
             FC_TICK(4);
             if (!ALIAS) pending = (next < total_tiles) ? stage(second_n, row_n, tcol_n) : false;
-            if (act) {
-                if (!split4) {
+            // Rows ky = 0 and ky = N/2 of a real column transform are real: they share the
+            // scratch row 0 as (re, im) and are transformed together in step 3.
+            if (!split4) {
+                if (gA < gcount) {
                     float2* dst = sMid + gA * P + cA;
-                    static_for<NC>([&](auto Kk) {
-                        constexpr int k = decltype(Kk)::value;
-                        dst[k * PW] = make_float2(Xr[k], Xi[k]);
-                    });
-                } else {
-                    float2* dst = sMid + g4 * P + c4 + q4 * PW;
-                    static_for<L>([&](auto Kk) {
-                        constexpr int k = decltype(Kk)::value;
-                        if (4 * k + q4 <= M) dst[4 * k * PW] = make_float2(br[k], bi[k]);
-                    });
+                    if (act) {
+                        dst[0] = make_float2(Xr[0], Xr[M]);
+                        static_for<M - 1>([&](auto Kk) {
+                            constexpr int k = decltype(Kk)::value + 1;
+                            dst[k * PW] = make_float2(Xr[k], Xi[k]);
+                        });
+                    } else if (!narrow) {
+                        // idle lanes zero the columns past the plane, so that step 3 reads
+                        // whole rows without a test per element
+                        static_for<M>([&](auto Kk) {
+                            constexpr int k = decltype(Kk)::value;
+                            dst[k * PW] = make_float2(0.0f, 0.0f);
+                        });
+                    }
                 }
+            } else if (act) {
+                float2* dst = sMid + g4 * P + c4 + q4 * PW;
+                if (q4 == 0) bi[0] = br[L / 2];     // ky = N/2 sits at k = N/8 of quarter 0
+                static_for<L>([&](auto Kk) {
+                    constexpr int k = decltype(Kk)::value;
+                    if (4 * k + q4 < M) dst[4 * k * PW] = make_float2(br[k], bi[k]);
+                });
             }
         }
         FC_TICK(5);
@@ -405,16 +462,16 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             float ar[M], ai[M];
             const float2* rowp = sMid + gB * P + kyp * PW;
             const bool packed = (kyp == 0);
-            auto load = [&](auto Cc) -> float2 {
-                constexpr int c = decltype(Cc)::value;
-                float2 v;
-                if (c >= w) return make_float2(0.0f, 0.0f);   // columns the tile never wrote
-                v = rowp[c];
-                if (packed) v.y = rowp[M * PW + c].x;   // row ky = N/2 rides as the imaginary part
-                return v;
-            };
-            if (q == 0) load_split<N, false, 0>(load, ar, ai);
-            else        load_split<N, false, 1>(load, ar, ai);
+            auto load = [&](auto Cc) -> float2 { return rowp[decltype(Cc)::value]; };
+            if (narrow) {
+                // at most N/2 live columns: the other half of every butterfly is zero
+                if (q == 0) load_split_narrow<N, false, 0>(load, w, ar, ai);
+                else        load_split_narrow<N, false, 1>(load, w, ar, ai);
+            } else {
+                // every column of the scratch row is valid (zeros past the plane)
+                if (q == 0) load_split<N, false, 0>(load, ar, ai);
+                else        load_split<N, false, 1>(load, ar, ai);
+            }
             FC_TICK(7);
             if constexpr (TMA && SALIAS) __syncthreads();   // scratch consumed: it becomes the staging tile
             FC_TICK(8);
@@ -630,15 +687,12 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
         }
         if (TMA || gB < gcount) {
             cfft<M, true>(ar, ai);  // ar/ai[m] = value at column c = 2m+q
+            // the packed row comes out as (row ky = 0, row ky = N/2) in (re, im): it stays
+            // packed in scratch row 0 and step 2 takes it apart
             float2* dst = sMid + gB * P + kyp * PW + q;
             static_for<M>([&](auto Mm) {
                 constexpr int m = decltype(Mm)::value;
-                if (!packed) {
-                    dst[2 * m] = make_float2(ar[m], ai[m]);
-                } else {
-                    dst[2 * m] = make_float2(ar[m], 0.0f);
-                    dst[M * PW + 2 * m] = make_float2(ai[m], 0.0f);
-                }
+                dst[2 * m] = make_float2(ar[m], ai[m]);
             });
         }
         __syncthreads();
@@ -650,26 +704,30 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             {
                 float Xr[NC], Xi[NC];
                 const float2* src = sMid + gA * P + cA;
-                static_for<NC>([&](auto Kk) {
+                static_for<M>([&](auto Kk) {
                     constexpr int k = decltype(Kk)::value;
                     const float2 t = src[k * PW];
-                    Xr[k] = t.x; Xi[k] = t.y;
+                    if constexpr (k == 0) {
+                        Xr[0] = t.x; Xi[0] = 0.0f; Xr[M] = t.y; Xi[M] = 0.0f;
+                    } else {
+                        Xr[k] = t.x; Xi[k] = t.y;
+                    }
                 });
                 irfft<N>(Xr, Xi, v);
             }
+            // the crop is the first hc rows: one running pointer, one uniform test per row
             float* dst = p.real_out + ((size_t)row * p.C + c0 + gA) * hw + cA;
             const float scale = p.scale;
-            if (!p.accumulate) {
-                static_for<N>([&](auto Rr) {
-                    constexpr int r = decltype(Rr)::value;
-                    if (r < hc) dst[r * wc] = v[r] * scale;
-                });
-            } else {
-                static_for<N>([&](auto Rr) {
-                    constexpr int r = decltype(Rr)::value;
-                    if (r < hc) dst[r * wc] = fc_fma(v[r], scale, dst[r * wc]);
-                });
-            }
+            const bool acc = p.accumulate != 0;
+            static_for<N>([&](auto Rr) {
+                constexpr int r = decltype(Rr)::value;
+                if (r < hc) {
+                    float o = v[r] * scale;
+                    if (acc) o += *dst;
+                    *dst = o;
+                    dst += wc;
+                }
+            });
         }
     }
 }
