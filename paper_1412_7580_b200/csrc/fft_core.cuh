@@ -272,4 +272,166 @@ FC_HD void dif_split(const float (&xr)[N], const float (&xi)[N], float (&ar)[N /
     });
 }
 
+// ---------------------------------------------------------------------------
+// Real-input FFT of length N split over two cooperating threads.  Both threads
+// see all N samples; thread Q in {0,1} returns the bins k = 2i + Q of the
+// Hermitian half 0..N/2 in O[i]: Q = 0 gets k = 0, 2, .., N/2 (N/4 + 1 bins),
+// Q = 1 gets k = 1, 3, .., N/2 - 1 (N/4 bins, O[N/4] untouched).
+// With z_j = x_2j + i x_2j+1 (M = N/2 points) the thread takes one
+// decimation-in-frequency step, a_j = z_j +- z_{j+M/2} (times w_M^j for Q = 1),
+// and an M/2-point FFT, which yields Z_{2m+Q}; the Hermitian post-pass of rfft
+// pairs Z_k with Z_{M-k}, and k and M-k have the same parity, so it stays inside
+// the thread.
+// ---------------------------------------------------------------------------
+template <int N, int Q, class Load>
+FC_HD void rfft_half(Load&& x, float (&Or)[N / 4 + 1], float (&Oi)[N / 4 + 1]) {
+    static_assert(N >= 8, "needs an even quarter length");
+    constexpr int M = N / 2, H = M / 2;
+    float ar[H], ai[H];
+    static_for<H>([&](auto J) {
+        constexpr int j = decltype(J)::value;
+        const float lr = x(std::integral_constant<int, 2 * j>{});
+        const float li = x(std::integral_constant<int, 2 * j + 1>{});
+        const float hr = x(std::integral_constant<int, 2 * j + M>{});
+        const float hi = x(std::integral_constant<int, 2 * j + M + 1>{});
+        if constexpr (Q == 0) {
+            ar[j] = lr + hr; ai[j] = li + hi;
+        } else {
+            const float dr = lr - hr, di = li - hi;
+            if constexpr (j == 0) {
+                ar[j] = dr; ai[j] = di;
+            } else if constexpr (4 * j == M) {
+                ar[j] = di; ai[j] = -dr;
+            } else {
+                constexpr float c = Tw<M, j>::c, s = Tw<M, j>::s;
+                ar[j] = fc_fma(s, di, c * dr);
+                ai[j] = fc_fma(-s, dr, c * di);
+            }
+        }
+    });
+    cfft<H, false>(ar, ai);                       // ar/ai[m] = Z_{2m+Q}
+    auto pair = [&](auto K) {                     // bins k and M-k from Z_k and Z_{M-k}
+        constexpr int k = decltype(K)::value;
+        constexpr int m = (k - Q) / 2, mp = (M - k - Q) / 2;
+        constexpr float hc = 0.5f * Tw<N, k>::c;
+        constexpr float hs = 0.5f * Tw<N, k>::s;
+        const float pr = ar[m], pi = ai[m], qr = ar[mp], qi = ai[mp];
+        const float er = pr + qr, ei = pi - qi;       // 2 E_k
+        const float orr = pi + qi, oi = qr - pr;      // 2 O_k
+        const float tr = fc_fma(hs, oi, hc * orr);
+        const float ti = fc_fma(-hs, orr, hc * oi);
+        Or[m] = fc_fma(0.5f, er, tr);
+        Oi[m] = fc_fma(0.5f, ei, ti);
+        Or[mp] = fc_fma(0.5f, er, -tr);
+        Oi[mp] = fc_fma(-0.5f, ei, ti);
+    };
+    if constexpr (Q == 0) {
+        Or[0] = ar[0] + ai[0]; Oi[0] = 0.0f;          // k = 0
+        Or[H] = ar[0] - ai[0]; Oi[H] = 0.0f;          // k = M
+        Or[H / 2] = ar[H / 2]; Oi[H / 2] = -ai[H / 2];  // k = M/2
+        static_for<H / 2 - 1>([&](auto I) {            // k = 2, 4, .., M/2 - 2
+            pair(std::integral_constant<int, 2 * (decltype(I)::value + 1)>{});
+        });
+    } else {
+        static_for<H / 2>([&](auto I) {                // k = 1, 3, .., M/2 - 1
+            pair(std::integral_constant<int, 2 * decltype(I)::value + 1>{});
+        });
+    }
+}
+
+// ---------------------------------------------------------------------------
+// One radix-4 decimation-in-frequency step of an N-point complex transform split
+// over four cooperating threads.  All threads see the N inputs through load(j)
+// (a float2); thread Q in {0..3} forms the N/4 inputs of the quarter-size
+// transform whose outputs are X_{4m+Q}:
+//   a_j = (x_j + u^Q x_{j+L} + u^2Q x_{j+2L} + u^3Q x_{j+3L}) w_N^{+-Qj},  L = N/4,
+// with u = -i forward and +i inverse.
+// ---------------------------------------------------------------------------
+template <int N, bool INV, int Q, int J>
+FC_HD void split4_elem(const float2 x0, const float2 x1, const float2 x2, const float2 x3, float& outr,
+                       float& outi) {
+    float tr, ti;
+    if constexpr (Q == 0) {
+        tr = (x0.x + x2.x) + (x1.x + x3.x); ti = (x0.y + x2.y) + (x1.y + x3.y);
+    } else if constexpr (Q == 2) {
+        tr = (x0.x + x2.x) - (x1.x + x3.x); ti = (x0.y + x2.y) - (x1.y + x3.y);
+    } else {
+        const float dr = x0.x - x2.x, di = x0.y - x2.y;     // x_j - x_{j+2L}
+        const float er = x1.x - x3.x, ei = x1.y - x3.y;     // x_{j+L} - x_{j+3L}
+        // forward Q = 1 (inverse Q = 3): d - i e;   forward Q = 3 (inverse Q = 1): d + i e
+        if constexpr ((Q == 1) != INV) { tr = dr + ei; ti = di - er; }
+        else                           { tr = dr - ei; ti = di + er; }
+    }
+    if constexpr (Q == 0 || J == 0) {
+        outr = tr; outi = ti;
+    } else {
+        constexpr float c = Tw<N, Q * J>::c;
+        constexpr float s = INV ? -Tw<N, Q * J>::s : Tw<N, Q * J>::s;
+        // w = (c, -s): w t = (c tr + s ti, c ti - s tr)
+        outr = fc_fma(s, ti, c * tr);
+        outi = fc_fma(-s, tr, c * ti);
+    }
+}
+template <int N, bool INV, int Q, class Load>
+FC_HD void load_split4(Load&& load, float (&ar)[N / 4], float (&ai)[N / 4]) {
+    constexpr int L = N / 4;
+    static_for<L>([&](auto J) {
+        constexpr int j = decltype(J)::value;
+        const float2 x0 = load(J), x1 = load(std::integral_constant<int, j + L>{});
+        const float2 x2 = load(std::integral_constant<int, j + 2 * L>{});
+        const float2 x3 = load(std::integral_constant<int, j + 3 * L>{});
+        split4_elem<N, INV, Q, j>(x0, x1, x2, x3, ar[j], ai[j]);
+    });
+}
+
+// ---------------------------------------------------------------------------
+// Inverse of the real-input FFT split over two cooperating threads (decimation
+// in time).  Thread Q in {0,1} reads the bins k = Q (mod 2) of the Hermitian half
+// through X(k) (a float2; X(0) must return (Re X_0, Re X_{N/2}) -- both bins are
+// real), forms Z'_{2m+Q} with the pre-pass of irfft (k and M-k have the same
+// parity) and runs an M/2-point inverse FFT.  Result: Q = 0 returns E_j, Q = 1
+// returns w_M^{-j} O_j (j < M/2); then z_j = E_j + w^{-j} O_j and
+// z_{j+M/2} = E_j - w^{-j} O_j, with x_2j = Re z_j, x_2j+1 = Im z_j (times N).
+// ---------------------------------------------------------------------------
+template <int N, int Q, class LoadX>
+FC_HD void irfft_half(LoadX&& X, float (&er)[N / 4], float (&ei)[N / 4]) {
+    static_assert(N >= 8, "needs an even quarter length");
+    constexpr int M = N / 2, H = M / 2;
+    auto pair = [&](auto K) {
+        constexpr int k = decltype(K)::value;
+        constexpr int m = (k - Q) / 2, mp = (M - k - Q) / 2;
+        constexpr float c = Tw<N, k>::c, s = Tw<N, k>::s;
+        const float2 P = X(K), Qv = X(std::integral_constant<int, M - k>{});
+        const float sr = P.x + Qv.x, si = P.y - Qv.y;   // P + conj Q
+        const float dr = P.x - Qv.x, di = P.y + Qv.y;   // P - conj Q
+        const float ur = fc_fma(-s, di, c * dr);        // w_N^{-k} D
+        const float ui = fc_fma(s, dr, c * di);
+        er[m] = sr - ui;  ei[m] = si + ur;
+        er[mp] = sr + ui; ei[mp] = ur - si;
+    };
+    if constexpr (Q == 0) {
+        const float2 dc = X(std::integral_constant<int, 0>{});
+        er[0] = dc.x + dc.y; ei[0] = dc.x - dc.y;
+        const float2 mid = X(std::integral_constant<int, H>{});
+        er[H / 2] = 2.0f * mid.x; ei[H / 2] = -2.0f * mid.y;
+        static_for<H / 2 - 1>([&](auto I) {
+            pair(std::integral_constant<int, 2 * (decltype(I)::value + 1)>{});
+        });
+    } else {
+        static_for<H / 2>([&](auto I) {
+            pair(std::integral_constant<int, 2 * decltype(I)::value + 1>{});
+        });
+    }
+    cfft<H, true>(er, ei);
+    if constexpr (Q == 1) {
+        static_for<H - 1>([&](auto J) {
+            constexpr int j = decltype(J)::value + 1;
+            constexpr float c = Tw<M, j>::c, s = Tw<M, j>::s;
+            const float a = er[j], b = ei[j];
+            er[j] = fc_fma(-s, b, c * a);
+            ei[j] = fc_fma(s, a, c * b);
+        });
+    }
+}
+
 }  // namespace fc

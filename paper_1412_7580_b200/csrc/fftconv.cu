@@ -14,6 +14,7 @@
 #include "cgemm_ffma.cuh"
 #include "cgemm_tc.cuh"
 #include "fft_kernels.cuh"
+#include "fft_big.cuh"
 
 #define FFTCONV_API extern "C" __attribute__((visibility("default")))
 
@@ -114,6 +115,26 @@ size_t pass_bytes(const conv_plan_s& p, int pass) {
            align_up(d.c.spec.bytes(p.bins), kAlign);
 }
 
+// Bytes of the spectra regions (with the header); the scratch of the two-pass transforms
+// (n = 128) follows them.
+size_t spectra_bytes(const conv_plan_s* plan) {
+    if (plan->reuse) {
+        // one region per tensor family plus one for the result spectrum of the running pass
+        const PassDesc d = describe(*plan, PASS_FPROP);      // a = x, b = w, c = y
+        const size_t bx = align_up(d.a.spec.bytes(plan->bins), kAlign),
+                     bw = align_up(d.b.spec.bytes(plan->bins), kAlign),
+                     by = align_up(d.c.spec.bytes(plan->bins), kAlign);
+        const size_t br = bx > bw ? (bx > by ? bx : by) : (bw > by ? bw : by);
+        return kHeaderBytes + bx + bw + by + br;
+    }
+    size_t m = 0;
+    for (int pass = 0; pass < 3; ++pass) {
+        size_t b = pass_bytes(*plan, pass);
+        if (b > m) m = b;
+    }
+    return kHeaderBytes + m;
+}
+
 bool valid_n(int n) { return n == 8 || n == 16 || n == 32 || n == 64 || n == 128; }
 
 int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, float* c_out,
@@ -160,27 +181,34 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     };
     const bool timing = plan->timing && plan->ev_made;
     auto mark = [&](int i) { if (timing) cudaEventRecord(plan->ev[i], st); };
+    // n = 128 runs the two-pass transforms (one launch per operand, scratch behind the spectra)
+    const bool big = fc::big_scratch_bytes(plan->n) != 0;
+    float* scratch = reinterpret_cast<float*>(base + align_up(spectra_bytes(plan), kAlign));
+    const size_t scratch_bytes = fc::big_scratch_bytes(plan->n);
+    auto forward = [&](const fc::FftParams& pa, const fc::FftParams* pb) -> cudaError_t {
+        g_launches.fetch_add((big && pb) ? 2 : 1, std::memory_order_relaxed);
+        if (!big) return fc::launch_r2c<true>(plan->n, pa, pb, st);
+        cudaError_t e = fc::launch_r2c_big<128>(pa, scratch, scratch_bytes, st);
+        if (e == cudaSuccess && pb) e = fc::launch_r2c_big<128>(*pb, scratch, scratch_bytes, st);
+        return e;
+    };
     mark(0);
     const fc::FftParams fa = operand(d.a, a_in, specA), fb = operand(d.b, b_in, specB);
     if (!need_a || !need_b) {
         // spectrum reuse: at most one operand left to transform
         if (need_a || need_b) {
-            g_launches.fetch_add(1, std::memory_order_relaxed);
-            if (fc::launch_r2c<true>(plan->n, need_a ? fa : fb, nullptr, st) != cudaSuccess)
-                return FFTCONV_ECUDA;
+            if (forward(need_a ? fa : fb, nullptr) != cudaSuccess) return FFTCONV_ECUDA;
         }
         mark(1);
     } else if (!timing || plan->timing == 1) {
         // both forward transforms in one launch: one ramp-up, one tail
-        g_launches.fetch_add(1, std::memory_order_relaxed);
-        if (fc::launch_r2c<true>(plan->n, fa, &fb, st) != cudaSuccess) return FFTCONV_ECUDA;
+        if (forward(fa, &fb) != cudaSuccess) return FFTCONV_ECUDA;
         mark(1);
     } else {
         // timing mode 2: one kernel per operand, to time the two transforms apart
-        g_launches.fetch_add(2, std::memory_order_relaxed);
-        if (fc::launch_r2c<true>(plan->n, fa, nullptr, st) != cudaSuccess) return FFTCONV_ECUDA;
+        if (forward(fa, nullptr) != cudaSuccess) return FFTCONV_ECUDA;
         mark(1);
-        if (fc::launch_r2c<true>(plan->n, fb, nullptr, st) != cudaSuccess) return FFTCONV_ECUDA;
+        if (forward(fb, nullptr) != cudaSuccess) return FFTCONV_ECUDA;
     }
     mark(2);
 
@@ -203,7 +231,9 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     ip.scale = 1.0f / ((float)plan->n * (float)plan->n);
     ip.accumulate = accumulate ? 1 : 0;
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    if (fc::launch_c2r<true>(plan->n, ip, st) != cudaSuccess) return FFTCONV_ECUDA;
+    if ((big ? fc::launch_c2r_big<128>(ip, scratch, scratch_bytes, st)
+             : fc::launch_c2r<true>(plan->n, ip, st)) != cudaSuccess)
+        return FFTCONV_ECUDA;
     mark(4);
     if (timing) plan->timed = true;
     return FFTCONV_OK;
@@ -261,21 +291,7 @@ FFTCONV_API int conv_plan_pass_math(const conv_plan_t* plan, int pass) {
 
 FFTCONV_API size_t conv_plan_workspace_bytes(const conv_plan_t* plan) {
     if (!plan) return 0;
-    if (plan->reuse) {
-        // one region per tensor family plus one for the result spectrum of the running pass
-        const PassDesc d = describe(*plan, PASS_FPROP);      // a = x, b = w, c = y
-        const size_t bx = align_up(d.a.spec.bytes(plan->bins), kAlign),
-                     bw = align_up(d.b.spec.bytes(plan->bins), kAlign),
-                     by = align_up(d.c.spec.bytes(plan->bins), kAlign);
-        const size_t br = bx > bw ? (bx > by ? bx : by) : (bw > by ? bw : by);
-        return kHeaderBytes + bx + bw + by + br;
-    }
-    size_t m = 0;
-    for (int pass = 0; pass < 3; ++pass) {
-        size_t b = pass_bytes(*plan, pass);
-        if (b > m) m = b;
-    }
-    return kHeaderBytes + m;
+    return align_up(spectra_bytes(plan), kAlign) + fc::big_scratch_bytes(plan->n);
 }
 
 FFTCONV_API int conv_plan_set_workspace(conv_plan_t* plan, void* dev_ptr, size_t bytes) {

@@ -59,6 +59,9 @@ SMALL = [
     (3, 4, 1, 57, 57, 3, 3, 64),
     (1, 2, 3, 128, 128, 13, 13, 128),
     (2, 3, 2, 120, 120, 5, 5, 128),
+    (3, 9, 10, 128, 128, 7, 7, 128),    # two-pass transforms: a full tile of 8 planes and a ragged one
+    (2, 5, 3, 97, 101, 5, 9, 128),      # plane sizes that break the 16-byte alignment of the plane copies
+    (1, 17, 12, 120, 121, 13, 3, 128),
     (16, 16, 16, 13, 13, 3, 3, 16),
     (1, 64, 1, 16, 16, 5, 5, 16),
 ]
@@ -85,6 +88,25 @@ def test_accgrad_accumulates():
     import paper_1412_7580_b200 as fc
     from paper_1412_7580_b200 import workloads as wl
     s = wl.ConvShape("acc", 4, 6, 5, 13, 13, 3, 3, 16, cfg=7, point=1)
+    x, dy = wl.make_x(s), wl.make_dy(s)
+    init = wl.make_w(s)
+    p = fc.conv_plan(*s.args())
+    fc.conv_plan_set_math(p, fc.MATH_FP32)
+    fc.conv_plan_alloc_workspace(p)
+    dw = torch.from_numpy(init.copy()).cuda()
+    fc.conv_accgrad(p, torch.from_numpy(dy).cuda(), torch.from_numpy(x).cuda(), dw, accumulate=True)
+    torch.cuda.synchronize()
+    ref = init.astype(np.float64) + oracle.accgrad(dy, x, s.kh, s.kw)
+    assert relerr(dw.cpu().numpy().astype(np.float64), ref) <= 1e-4
+
+
+def test_accgrad_accumulates_two_pass_transforms():
+    """accumulate = 1 through the n = 128 inverse transform."""
+    import torch
+    import oracle
+    import paper_1412_7580_b200 as fc
+    from paper_1412_7580_b200 import workloads as wl
+    s = wl.ConvShape("acc128", 2, 9, 3, 120, 120, 7, 7, 128, cfg=7, point=2)
     x, dy = wl.make_x(s), wl.make_dy(s)
     init = wl.make_w(s)
     p = fc.conv_plan(*s.args())
