@@ -284,10 +284,9 @@ FC_HD void dif_split(const float (&xr)[N], const float (&xi)[N], float (&ar)[N /
 // the thread.
 // ---------------------------------------------------------------------------
 template <int N, int Q, class Load>
-FC_HD void rfft_half(Load&& x, float (&Or)[N / 4 + 1], float (&Oi)[N / 4 + 1]) {
+FC_HD void rfft_half_split(Load&& x, float (&ar)[N / 4], float (&ai)[N / 4]) {
     static_assert(N >= 8, "needs an even quarter length");
     constexpr int M = N / 2, H = M / 2;
-    float ar[H], ai[H];
     static_for<H>([&](auto J) {
         constexpr int j = decltype(J)::value;
         const float lr = x(std::integral_constant<int, 2 * j>{});
@@ -309,6 +308,12 @@ FC_HD void rfft_half(Load&& x, float (&Or)[N / 4 + 1], float (&Oi)[N / 4 + 1]) {
             }
         }
     });
+}
+// Second half of rfft_half: the N/4-point FFT and the Hermitian post-pass; every bin is
+// handed to emit(i, re, im) with i a compile-time index (bin k = 2i + Q) as soon as it exists.
+template <int N, int Q, class Emit>
+FC_HD void rfft_half_finish(float (&ar)[N / 4], float (&ai)[N / 4], Emit&& emit) {
+    constexpr int M = N / 2, H = M / 2;
     cfft<H, false>(ar, ai);                       // ar/ai[m] = Z_{2m+Q}
     auto pair = [&](auto K) {                     // bins k and M-k from Z_k and Z_{M-k}
         constexpr int k = decltype(K)::value;
@@ -320,15 +325,13 @@ FC_HD void rfft_half(Load&& x, float (&Or)[N / 4 + 1], float (&Oi)[N / 4 + 1]) {
         const float orr = pi + qi, oi = qr - pr;      // 2 O_k
         const float tr = fc_fma(hs, oi, hc * orr);
         const float ti = fc_fma(-hs, orr, hc * oi);
-        Or[m] = fc_fma(0.5f, er, tr);
-        Oi[m] = fc_fma(0.5f, ei, ti);
-        Or[mp] = fc_fma(0.5f, er, -tr);
-        Oi[mp] = fc_fma(-0.5f, ei, ti);
+        emit(std::integral_constant<int, m>{}, fc_fma(0.5f, er, tr), fc_fma(0.5f, ei, ti));
+        emit(std::integral_constant<int, mp>{}, fc_fma(0.5f, er, -tr), fc_fma(-0.5f, ei, ti));
     };
     if constexpr (Q == 0) {
-        Or[0] = ar[0] + ai[0]; Oi[0] = 0.0f;          // k = 0
-        Or[H] = ar[0] - ai[0]; Oi[H] = 0.0f;          // k = M
-        Or[H / 2] = ar[H / 2]; Oi[H / 2] = -ai[H / 2];  // k = M/2
+        emit(std::integral_constant<int, 0>{}, ar[0] + ai[0], 0.0f);          // k = 0
+        emit(std::integral_constant<int, H>{}, ar[0] - ai[0], 0.0f);          // k = M
+        emit(std::integral_constant<int, H / 2>{}, ar[H / 2], -ai[H / 2]);    // k = M/2
         static_for<H / 2 - 1>([&](auto I) {            // k = 2, 4, .., M/2 - 2
             pair(std::integral_constant<int, 2 * (decltype(I)::value + 1)>{});
         });
@@ -337,6 +340,15 @@ FC_HD void rfft_half(Load&& x, float (&Or)[N / 4 + 1], float (&Oi)[N / 4 + 1]) {
             pair(std::integral_constant<int, 2 * decltype(I)::value + 1>{});
         });
     }
+}
+template <int N, int Q, class Load>
+FC_HD void rfft_half(Load&& x, float (&Or)[N / 4 + 1], float (&Oi)[N / 4 + 1]) {
+    float ar[N / 4], ai[N / 4];
+    rfft_half_split<N, Q>(static_cast<Load&&>(x), ar, ai);
+    rfft_half_finish<N, Q>(ar, ai, [&](auto I, float re, float im) {
+        Or[decltype(I)::value] = re;
+        Oi[decltype(I)::value] = im;
+    });
 }
 
 // ---------------------------------------------------------------------------
