@@ -35,8 +35,8 @@ FP32_FFMA_TFLOPS_NOMINAL = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x lanes x 2 fl
 # keyed by (workload, kernel, pass); None where no capture exists.
 NCU_TRAFFIC = {
     ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "bprop"): 291.9e6,
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "accgrad"): 287.2e6,
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "fprop"): 156.6e6,
+    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "accgrad"): 287.4e6,
+    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "fprop"): 157.2e6,
 }
 
 
@@ -279,8 +279,11 @@ def run_ours(args, s):
         step(); reps += 1
     torch.cuda.synchronize()
     t1 = time.time()
-    launches = 9 * args.steps          # per pass: both forward FFTs (one launch), contraction, inverse FFT
-    assert fc.fftconv_launch_count() - launches0 == 9 * (args.steps + reps)
+    # counted by the library.  Per pass: the forward FFTs (one launch for both operands with the
+    # one-pass kernels, one per operand with the two-pass kernels), the contraction, the inverse FFT
+    counted = fc.fftconv_launch_count() - launches0
+    assert counted % (args.steps + reps) == 0 and counted // (args.steps + reps) in (9, 12)
+    launches = counted // (args.steps + reps) * args.steps
     clocks = sampler.stop(t0, t1) if rank == 0 else None
     ms_step = ms_total / args.steps
 
@@ -379,9 +382,11 @@ def run_ours(args, s):
             fc.conv_accgrad(plan_r, dyd, xd, dw)
         for _ in range(3):
             step_r()
+        lr0 = fc.fftconv_launch_count()
         ms_r = timed(step_r, args.steps) / args.steps
+        launches_r = (fc.fftconv_launch_count() - lr0) // args.steps
         reuse = {"ms_per_step": ms_r, "value": world * flops_step / (ms_r * 1e-3) / 1e9, "unit": UNIT,
-                 "gpu_launches_per_step": 8, "workspace_bytes": int(ws_r.numel()),
+                 "gpu_launches_per_step": launches_r, "workspace_bytes": int(ws_r.numel()),
                  "note": "x, w, dy spectra computed once per step and shared by the three passes"}
         fc.conv_plan_destroy(plan_r)
         del ws_r
@@ -423,6 +428,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=1, help="0 tiny, 1 mid (default), 2 large-kernel, 3 deep")
+    ap.add_argument("--shape", default=None,
+                    help="S,f,fp,h,w,kh,kw,n : a layer shape of your own instead of --config "
+                         "(seeded inputs as in the sweep; used for profiling single shapes)")
     ap.add_argument("--math", default="auto", choices=["auto", "fp32", "tf32"])
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -431,6 +439,11 @@ def main():
     args = ap.parse_args()
     from paper_1412_7580_b200 import workloads as wl
     s = wl.CONFIGS[args.config]
+    if args.shape:
+        dims = [int(v) for v in args.shape.split(",")]
+        assert len(dims) == 8, "--shape wants S,f,fp,h,w,kh,kw,n"
+        s = wl.ConvShape("custom_S%d_f%d_fp%d_%dx%d_k%dx%d_n%d" % tuple(dims), *dims, cfg=6,
+                         point=sum(dims), w_dist="fan_in", dy_dist="normal")
     if args.impl == "reference":
         run_reference(args, s)
     else:

@@ -35,34 +35,44 @@
 // the team's buffer, cropped / scaled / accumulated stores).
 #pragma once
 
+#include <stdlib.h>
+
 #include "fft_kernels.cuh"
 
 namespace fc {
 
 constexpr int BIG_G = 8;          // planes per tile
-constexpr int BIG_TEAM = 256;     // threads per team
-constexpr int BIG_T = 2 * BIG_TEAM;  // threads per CTA
-constexpr int BIG_KC = 8;         // rows ky per chunk
-constexpr int BIG_MAX_CTAS = 160; // scratch is sized for this many CTAs
+constexpr int BIG_MAX_SMS = 160;  // scratch is sized for this many SMs
+
+// teams per CTA and CTAs per SM the kernels are built for
+template <int N> struct BigCfg;
+template <> struct BigCfg<128> { static constexpr int NT = 2, MINB = 1; };
+template <> struct BigCfg<64>  { static constexpr int NT = 4, MINB = 2; };
 
 template <int N>
 struct BigGeom {
     static constexpr int M = N / 2, NC = M + 1, L = N / 4, H = N / 4;
-    static constexpr int ROWS = BIG_KC * BIG_G;                  // rows per chunk
+    static constexpr int TEAM = 2 * N;                           // threads per team
+    static constexpr int ROWS = N / 2;                           // rows per chunk (four threads per row)
+    static constexpr int KC = ROWS / BIG_G;                      // rows ky per chunk
     static constexpr int PITCH = N + 2;                          // float2 per row: 16-byte multiple, odd in 16-byte units
     static constexpr size_t INBUF = (size_t)ROWS * PITCH * 8;
     static constexpr size_t STAGE = (size_t)2 * N * ROWS * 4;
     static constexpr size_t STAGE_NY = (size_t)2 * N * BIG_G * 4;
     static constexpr size_t PLANE = (size_t)N * N * 4;
     static constexpr size_t SCRATCH_PER_CTA = (size_t)BIG_G * M * N * 8;
-    static constexpr size_t SMEM = 2 * INBUF + STAGE_NY;       // one buffer per team + the ky = N/2 staging
+    static constexpr int NT = BigCfg<N>::NT;                     // teams per CTA
+    static constexpr int THREADS = NT * TEAM;
+    static constexpr size_t SMEM = NT * INBUF + STAGE_NY;      // one buffer per team + the ky = N/2 staging
     static_assert(PLANE <= INBUF && STAGE <= INBUF, "a team's buffer holds a plane, a chunk or a staging tile");
     static_assert((size_t)2 * H * N * 8 <= INBUF, "the exchange buffer fits a team's buffer");
-    static_assert(BIG_TEAM == 2 * N && BIG_TEAM == 4 * ROWS, "thread roles");
+    static_assert(TEAM == 4 * ROWS && KC >= 1 && M % KC == 0, "thread roles");
 };
 
 static inline size_t big_scratch_bytes(int n) {
-    return n == 128 ? (size_t)BIG_MAX_CTAS * BigGeom<128>::SCRATCH_PER_CTA : 0;
+    if (n == 128) return (size_t)BIG_MAX_SMS * BigCfg<128>::MINB * BigGeom<128>::SCRATCH_PER_CTA;
+    if (n == 64) return (size_t)BIG_MAX_SMS * BigCfg<64>::MINB * BigGeom<64>::SCRATCH_PER_CTA;
+    return 0;
 }
 
 // Planar spectrum [2][N][NC][R][ld] seen as a 4-D tensor (col, row, ky, part*N + kx):
@@ -173,8 +183,9 @@ __device__ __forceinline__ float2 big_ld2(const float2* a, uint64_t pol) {
     return __ldcg(a);
 #endif
 }
+template <int TEAM>
 __device__ __forceinline__ void big_team_sync(int team) {
-    asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "n"(BIG_TEAM) : "memory");
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "n"(TEAM) : "memory");
 }
 __device__ __forceinline__ void fk_cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int PENDING>
@@ -204,17 +215,17 @@ __device__ __forceinline__ void big_split4_rows(const float2* rowp, float (&ar)[
 // Forward.
 // ---------------------------------------------------------------------------
 template <int N>
-__global__ void __launch_bounds__(BIG_T, 1)
+__global__ void __launch_bounds__(BigGeom<N>::THREADS, BigCfg<N>::MINB)
 r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmNy,
                const FftParams p, float2* __restrict__ scratch_all) {
     using Gm = BigGeom<N>;
-    constexpr int M = Gm::M, L = Gm::L, H = Gm::H, G = BIG_G, T = BIG_TEAM, PITCH = Gm::PITCH;
+    constexpr int M = Gm::M, L = Gm::L, H = Gm::H, G = BIG_G, T = Gm::TEAM, NT = Gm::NT, KC = Gm::KC, PITCH = Gm::PITCH;
     extern __shared__ __align__(128) unsigned char fc_smem[];
     float2* scratch = scratch_all + (size_t)blockIdx.x * (G * M * N);
 
     const int team = threadIdx.x / T, tid = threadIdx.x - team * T;      // tid: index inside the team
     unsigned char* buf = fc_smem + (size_t)team * Gm::INBUF;            // the team's buffer
-    float* sNy = reinterpret_cast<float*>(fc_smem + 2 * Gm::INBUF);
+    float* sNy = reinterpret_cast<float*>(fc_smem + NT * Gm::INBUF);
     const int q2 = tid / N, cA = tid - q2 * N;             // step A: (half, column)
     const int q4 = tid / Gm::ROWS, rB = tid - q4 * Gm::ROWS;   // step B: (quarter, row = ky_local*8 + plane)
     const int h = p.h, w = p.w, hw = h * w;
@@ -240,7 +251,7 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
 #pragma unroll 4
         for (int i = tid; i < Gm::ROWS * PER_ROW; i += T) {
             const int rr = i / PER_ROW, pc = i - rr * PER_ROW;
-            const int g = rr & (G - 1), ky = ci * BIG_KC + (rr >> 3);
+            const int g = rr & (G - 1), ky = ci * KC + (rr >> 3);
             fk_cp16(fk_smem_u32(dst + rr * PITCH + 2 * pc), scratch + ((size_t)(g * M + ky) * N + 2 * pc), keep);
         }
     };
@@ -251,12 +262,12 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
         const int c0 = tcol * G;
         const int gcount = min(G, p.C - c0);
 
-        // ---- A: column transforms; planes team, team + 2, .. ----------------------------
+        // ---- A: column transforms; planes team, team + NT, .. ----------------------------
         if (team < gcount) issue_plane(row, c0, team);
         fk_cp_commit();
-        for (int g = team; g < gcount; g += 2) {
+        for (int g = team; g < gcount; g += NT) {
             fk_cp_wait<0>();
-            big_team_sync(team);                           // plane g has landed for the team
+            big_team_sync<T>(team);                           // plane g has landed for the team
             const float* pl = reinterpret_cast<const float*>(buf) + cA;
             float ar[H], ai[H];
             const bool live = cA < w;
@@ -268,8 +279,8 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 if (q2 == 0) rfft_half_split<N, 0>(x, ar, ai);
                 else         rfft_half_split<N, 1>(x, ar, ai);
             }
-            big_team_sync(team);                           // plane g is in registers: the buffer takes the next one
-            if (g + 2 < gcount) issue_plane(row, c0, g + 2);
+            big_team_sync<T>(team);                           // plane g is in registers: the buffer takes the next one
+            if (g + NT < gcount) issue_plane(row, c0, g + NT);
             fk_cp_commit();
             float2* dst = scratch + (size_t)(g * M) * N + cA;
             if (live) {
@@ -298,20 +309,20 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
         fk_cp_wait<0>();
         __syncthreads();                                   // the scratch is complete
 
-        // ---- B: row transforms; chunks team, team + 2, .. --------------------------------
-        constexpr int CHUNKS = M / BIG_KC;
-        for (int ci = team; ci < CHUNKS; ci += 2) {
+        // ---- B: row transforms; chunks team, team + NT, .. --------------------------------
+        constexpr int CHUNKS = M / KC;
+        for (int ci = team; ci < CHUNKS; ci += NT) {
             issue_chunk(ci);
             fk_cp_commit();
             fk_cp_wait<0>();
-            big_team_sync(team);                           // chunk ci has landed for the team
+            big_team_sync<T>(team);                           // chunk ci has landed for the team
             float ar[L], ai[L];
             const float2* rowp = reinterpret_cast<const float2*>(buf) + rB * PITCH;
             if (q4 == 0)      big_split4_rows<N, false, 0>(rowp, ar, ai);
             else if (q4 == 1) big_split4_rows<N, false, 1>(rowp, ar, ai);
             else if (q4 == 2) big_split4_rows<N, false, 2>(rowp, ar, ai);
             else              big_split4_rows<N, false, 3>(rowp, ar, ai);
-            big_team_sync(team);                           // the chunk is in registers: the buffer becomes the staging tile
+            big_team_sync<T>(team);                           // the chunk is in registers: the buffer becomes the staging tile
             cfft<L, false>(ar, ai);                        // ar/ai[m] = F[kx = 4m + q4]
             float* sStage = reinterpret_cast<float*>(buf);
             float* o = sStage + q4 * Gm::ROWS + rB;
@@ -323,7 +334,7 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
             if (ci == 0) {
                 // row 0 of every plane holds Z = FFT(X_0 + i X_{N/2}); take it apart:
                 // X_0[k] = (Z_k + conj Z_{-k}) / 2,  X_{N/2}[k] = (Z_k - conj Z_{-k}) / (2i)
-                big_team_sync(team);
+                big_team_sync<T>(team);
                 for (int it = tid; it < G * (M + 1); it += T) {
                     const int g = it & (G - 1), k = it >> 3, kp = (N - k) & (N - 1);
                     float* a = sStage + g;                 // ky_local = 0: row index = plane
@@ -339,15 +350,15 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            big_team_sync(team);
+            big_team_sync<T>(team);
             if (tid == 0) {
-                fk_tma_store_4d(&tmS, fk_smem_u32(sStage), c0, row, ci * BIG_KC, 0, stream);
+                fk_tma_store_4d(&tmS, fk_smem_u32(sStage), c0, row, ci * KC, 0, stream);
                 if (ci == 0) fk_tma_store_4d(&tmNy, fk_smem_u32(sNy), c0, row, M, 0, stream);
                 fk_bulk_commit();
                 fk_bulk_wait_read();                       // the buffer may be overwritten after this
             }
             store_pending = true;
-            big_team_sync(team);
+            big_team_sync<T>(team);
         }
         __syncthreads();                                   // both teams are done with the scratch
     }
@@ -358,18 +369,18 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
 // Inverse.
 // ---------------------------------------------------------------------------
 template <int N>
-__global__ void __launch_bounds__(BIG_T, 1)
+__global__ void __launch_bounds__(BigGeom<N>::THREADS, BigCfg<N>::MINB)
 c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmNy,
                const FftParams p, float2* __restrict__ scratch_all) {
     using Gm = BigGeom<N>;
-    constexpr int M = Gm::M, L = Gm::L, H = Gm::H, G = BIG_G, T = BIG_TEAM, PITCH = Gm::PITCH;
+    constexpr int M = Gm::M, L = Gm::L, H = Gm::H, G = BIG_G, T = Gm::TEAM, NT = Gm::NT, KC = Gm::KC, PITCH = Gm::PITCH;
     extern __shared__ __align__(128) unsigned char fc_smem[];
-    __shared__ __align__(8) unsigned long long bar_storage[2];
+    __shared__ __align__(8) unsigned long long bar_storage[NT];
     float2* scratch = scratch_all + (size_t)blockIdx.x * (G * M * N);
 
     const int team = threadIdx.x / T, tid = threadIdx.x - team * T;
     unsigned char* buf = fc_smem + (size_t)team * Gm::INBUF;
-    float* sNy = reinterpret_cast<float*>(fc_smem + 2 * Gm::INBUF);
+    float* sNy = reinterpret_cast<float*>(fc_smem + NT * Gm::INBUF);
     const uint32_t bar = fk_smem_u32(&bar_storage[team]);
     const int q2 = tid / N, cA = tid - q2 * N;
     const int q4 = tid / Gm::ROWS, rB = tid - q4 * Gm::ROWS;
@@ -377,7 +388,7 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
     const int tpr = p.tiles_per_row;
     const float scale = p.scale;
     const bool acc = p.accumulate != 0;
-    constexpr int CHUNKS = M / BIG_KC;
+    constexpr int CHUNKS = M / KC;
     const uint64_t keep = big_policy_keep(), stream = big_policy_stream();
 
     if (tid == 0) {
@@ -393,11 +404,11 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
         const int c0 = tcol * G;
         const int gcount = min(G, p.C - c0);
 
-        // ---- B: row transforms; chunks team, team + 2, .. --------------------------------
-        for (int ci = team; ci < CHUNKS; ci += 2) {
+        // ---- B: row transforms; chunks team, team + NT, .. --------------------------------
+        for (int ci = team; ci < CHUNKS; ci += NT) {
             if (tid == 0) {
                 fk_mbar_expect_tx(bar, (uint32_t)(Gm::STAGE + (ci == 0 ? Gm::STAGE_NY : 0)));
-                fk_tma_load_4d(fk_smem_u32(buf), &tmS, c0, row, ci * BIG_KC, 0, bar, stream);
+                fk_tma_load_4d(fk_smem_u32(buf), &tmS, c0, row, ci * KC, 0, bar, stream);
                 if (ci == 0) fk_tma_load_4d(fk_smem_u32(sNy), &tmNy, c0, row, M, 0, bar, stream);
             }
             if (!dead && !fk_mbar_wait(bar, phase)) dead = true;
@@ -412,7 +423,7 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                     st[kx * Gm::ROWS + g] = a - d;
                     st[(N + kx) * Gm::ROWS + g] = b + c;
                 }
-                big_team_sync(team);
+                big_team_sync<T>(team);
             }
             float ar[L], ai[L];
             {
@@ -426,7 +437,7 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 else if (q4 == 2) load_split4<N, true, 2>(load, ar, ai);
                 else              load_split4<N, true, 3>(load, ar, ai);
             }
-            big_team_sync(team);                           // staging tile in registers: the buffer takes the rows
+            big_team_sync<T>(team);                           // staging tile in registers: the buffer takes the rows
             cfft<L, true>(ar, ai);                         // ar/ai[m] = value at column 4m + q4
             float2* sRows = reinterpret_cast<float2*>(buf);
             float2* dst = sRows + rB * PITCH + q4;
@@ -434,22 +445,22 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 constexpr int m = decltype(Mm)::value;
                 dst[4 * m] = make_float2(ar[m], ai[m]);
             });
-            big_team_sync(team);
+            big_team_sync<T>(team);
             constexpr int PER_ROW = N / 2;
 #pragma unroll 4
             for (int i = tid; i < Gm::ROWS * PER_ROW; i += T) {
                 const int rr = i / PER_ROW, pc = i - rr * PER_ROW;
-                const int g = rr & (G - 1), ky = ci * BIG_KC + (rr >> 3);
+                const int g = rr & (G - 1), ky = ci * KC + (rr >> 3);
                 const float4 v = *reinterpret_cast<const float4*>(sRows + rr * PITCH + 2 * pc);
                 big_st4(reinterpret_cast<float4*>(scratch + ((size_t)(g * M + ky) * N + 2 * pc)), v, keep);
             }
-            big_team_sync(team);                           // the buffer is free for the next chunk
+            big_team_sync<T>(team);                           // the buffer is free for the next chunk
         }
         __syncthreads();                                   // the scratch is complete for this CTA
 
-        // ---- A: column transforms; planes team, team + 2, .. ------------------------------
+        // ---- A: column transforms; planes team, team + NT, .. ------------------------------
         float2* sX = reinterpret_cast<float2*>(buf);
-        for (int g = team; g < gcount; g += 2) {
+        for (int g = team; g < gcount; g += NT) {
             float er[H], ei[H];
             const float2* src = scratch + (size_t)(g * M) * N + cA;
             auto X = [&](auto K) -> float2 {
@@ -464,7 +475,7 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 constexpr int j = decltype(J)::value;
                 mine[j * N] = make_float2(er[j], ei[j]);
             });
-            big_team_sync(team);
+            big_team_sync<T>(team);
             if (cA < wc) {
                 float* out = p.real_out + ((size_t)row * p.C + c0 + g) * hw + cA;
                 // z_j = E_j + O'_j (rows 2j, 2j+1),  z_{j+H} = E_j - O'_j (rows N/2 + 2j, ...)
@@ -489,7 +500,7 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                     }
                 });
             }
-            big_team_sync(team);                           // exchange buffer free for the next plane
+            big_team_sync<T>(team);                           // exchange buffer free for the next plane
         }
         __syncthreads();                                   // both teams are done with the scratch
     }
@@ -505,16 +516,16 @@ static cudaError_t launch_r2c_big(FftParams p, float* scratch, size_t scratch_by
     CUtensorMap tm, tmny;
     memset(&tm, 0, sizeof(tm));
     memset(&tmny, 0, sizeof(tmny));
-    if (!big_make_map<N>(&tm, p.spec_out, p, BIG_KC) || !big_make_map<N>(&tmny, p.spec_out, p, 1))
+    if (!big_make_map<N>(&tm, p.spec_out, p, Gm::KC) || !big_make_map<N>(&tmny, p.spec_out, p, 1))
         return cudaErrorInvalidValue;
     auto kern = r2c_big_kernel<N>;
     int grid = 0;
-    cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), BIG_T, Gm::SMEM, p.num_tiles, &grid);
+    cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), Gm::THREADS, Gm::SMEM, p.num_tiles, &grid);
     if (e != cudaSuccess) return e;
     const long long fit = (long long)(scratch_bytes / Gm::SCRATCH_PER_CTA);
     if (fit < 1) return cudaErrorInvalidValue;
     if (grid > fit) grid = (int)fit;
-    kern<<<grid, BIG_T, Gm::SMEM, st>>>(tm, tmny, p, reinterpret_cast<float2*>(scratch));
+    kern<<<grid, Gm::THREADS, Gm::SMEM, st>>>(tm, tmny, p, reinterpret_cast<float2*>(scratch));
     return cudaGetLastError();
 }
 
@@ -525,18 +536,37 @@ static cudaError_t launch_c2r_big(FftParams p, float* scratch, size_t scratch_by
     CUtensorMap tm, tmny;
     memset(&tm, 0, sizeof(tm));
     memset(&tmny, 0, sizeof(tmny));
-    if (!big_make_map<N>(&tm, p.spec_in, p, BIG_KC) || !big_make_map<N>(&tmny, p.spec_in, p, 1))
+    if (!big_make_map<N>(&tm, p.spec_in, p, Gm::KC) || !big_make_map<N>(&tmny, p.spec_in, p, 1))
         return cudaErrorInvalidValue;
     auto kern = c2r_big_kernel<N>;
     constexpr size_t SMEM = Gm::SMEM;
     int grid = 0;
-    cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), BIG_T, SMEM, p.num_tiles, &grid);
+    cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), Gm::THREADS, SMEM, p.num_tiles, &grid);
     if (e != cudaSuccess) return e;
     const long long fit = (long long)(scratch_bytes / Gm::SCRATCH_PER_CTA);
     if (fit < 1) return cudaErrorInvalidValue;
     if (grid > fit) grid = (int)fit;
-    kern<<<grid, BIG_T, SMEM, st>>>(tm, tmny, p, reinterpret_cast<float2*>(scratch));
+    kern<<<grid, Gm::THREADS, SMEM, st>>>(tm, tmny, p, reinterpret_cast<float2*>(scratch));
     return cudaGetLastError();
+}
+
+// Which plane sizes take the two-pass kernels.  n = 64 can run on either family; the
+// environment variable FFTCONV_TWO_PASS_64 (0 / 1) overrides the default for measurements.
+static inline bool big_uses_two_pass(int n) {
+    if (n == 128) return true;
+    if (n != 64) return false;
+    static int on = -1;
+    if (on < 0) {
+        const char* e = getenv("FFTCONV_TWO_PASS_64");
+        on = e ? (atoi(e) != 0) : 0;
+    }
+    return on == 1;
+}
+static cudaError_t launch_r2c_two_pass(int n, const FftParams& p, float* scratch, size_t bytes, cudaStream_t st) {
+    return n == 128 ? launch_r2c_big<128>(p, scratch, bytes, st) : launch_r2c_big<64>(p, scratch, bytes, st);
+}
+static cudaError_t launch_c2r_two_pass(int n, const FftParams& p, float* scratch, size_t bytes, cudaStream_t st) {
+    return n == 128 ? launch_c2r_big<128>(p, scratch, bytes, st) : launch_c2r_big<64>(p, scratch, bytes, st);
 }
 
 }  // namespace fc

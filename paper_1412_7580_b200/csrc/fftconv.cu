@@ -181,15 +181,15 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     };
     const bool timing = plan->timing && plan->ev_made;
     auto mark = [&](int i) { if (timing) cudaEventRecord(plan->ev[i], st); };
-    // n = 128 runs the two-pass transforms (one launch per operand, scratch behind the spectra)
-    const bool big = fc::big_scratch_bytes(plan->n) != 0;
+    // large planes run the two-pass transforms (one launch per operand, scratch behind the spectra)
+    const bool big = fc::big_uses_two_pass(plan->n);
     float* scratch = reinterpret_cast<float*>(base + align_up(spectra_bytes(plan), kAlign));
     const size_t scratch_bytes = fc::big_scratch_bytes(plan->n);
     auto forward = [&](const fc::FftParams& pa, const fc::FftParams* pb) -> cudaError_t {
         g_launches.fetch_add((big && pb) ? 2 : 1, std::memory_order_relaxed);
         if (!big) return fc::launch_r2c<true>(plan->n, pa, pb, st);
-        cudaError_t e = fc::launch_r2c_big<128>(pa, scratch, scratch_bytes, st);
-        if (e == cudaSuccess && pb) e = fc::launch_r2c_big<128>(*pb, scratch, scratch_bytes, st);
+        cudaError_t e = fc::launch_r2c_two_pass(plan->n, pa, scratch, scratch_bytes, st);
+        if (e == cudaSuccess && pb) e = fc::launch_r2c_two_pass(plan->n, *pb, scratch, scratch_bytes, st);
         return e;
     };
     mark(0);
@@ -231,7 +231,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     ip.scale = 1.0f / ((float)plan->n * (float)plan->n);
     ip.accumulate = accumulate ? 1 : 0;
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    if ((big ? fc::launch_c2r_big<128>(ip, scratch, scratch_bytes, st)
+    if ((big ? fc::launch_c2r_two_pass(plan->n, ip, scratch, scratch_bytes, st)
              : fc::launch_c2r<true>(plan->n, ip, st)) != cudaSuccess)
         return FFTCONV_ECUDA;
     mark(4);
