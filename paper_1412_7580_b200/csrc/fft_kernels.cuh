@@ -226,6 +226,13 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
     constexpr int PW = MidGeom<N, G>::PW, P = MidGeom<N, G>::P;
     constexpr bool TMA = (LAYOUT == LAYOUT_FREQ_TMA);
     constexpr int D = tma_bins_per_box(N);
+    // The packed row (ky = 0 with ky = N/2) is taken apart either by the two threads that
+    // transformed it or, with the TMA staging, afterwards by the whole CTA (one more barrier,
+    // but no warp does more than the others).  Measured on B200: the CTA-wide form is 3-10 %
+    // faster per launch for N <= 32; at N = 64 (16-byte staging rows) it is faster too, except
+    // that the second large operand of accGrad then runs 40 % slower, so N = 64 keeps the
+    // thread-local form.
+    constexpr bool WIDE_UNTANGLE = TMA && N <= 32;
     static_assert(HALF % 32 == 0, "the two halves of a row transform must be warp-uniform");
     extern __shared__ __align__(128) unsigned char fc_smem[];
     float* sIn = reinterpret_cast<float*>(fc_smem);
@@ -491,7 +498,10 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
                     o = p.spec_out + (size_t)(q * NC + kyp) * mat + (size_t)row * p.ld + c0 + gB;
                     sb = mat; sp = (size_t)B * mat;
                 }
-                if (!packed) {
+                // With the TMA staging the packed row is written like any other row and taken
+                // apart afterwards by the whole CTA (below): the lanes that hold it then do no
+                // more work than the rest.
+                if (WIDE_UNTANGLE || !packed) {
                     static_for<M>([&](auto Kk) {
                         constexpr int k = decltype(Kk)::value;
                         o[(size_t)(2 * k * NC) * sb] = ar[k];
@@ -548,6 +558,24 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
         }
         FC_TICK(10);
         if constexpr (TMA) {
+            // Row ky = 0 of every plane holds Z = FFT(X_0 + i X_{N/2}) of the two real rows:
+            // X_0[k] = (Z_k + conj Z_{-k}) / 2,  X_{N/2}[k] = (Z_k - conj Z_{-k}) / (2i); one
+            // (plane, k <= N/2) pair per thread, each touching only its own four bins.
+            if constexpr (WIDE_UNTANGLE) {
+            __syncthreads();
+            for (int it = tid; it < G * (M + 1); it += T) {
+                const int g = it % G, k = it / G, kp = (N - k) & (N - 1);
+                float* a = sStage + g;
+                const int ik = k * NC * G, ip = kp * NC * G;
+                const float fr = a[ik], fi = a[B * G + ik], gr = a[ip], gi = a[B * G + ip];
+                const float x0r = 0.5f * (fr + gr), x0i = 0.5f * (fi - gi);
+                const float xnr = 0.5f * (fi + gi), xni = 0.5f * (gr - fr);
+                a[ik] = x0r;          a[B * G + ik] = x0i;
+                a[ip] = x0r;          a[B * G + ip] = -x0i;
+                a[ik + M * G] = xnr;  a[B * G + ik + M * G] = xni;
+                a[ip + M * G] = xnr;  a[B * G + ip + M * G] = -xni;
+            }
+            }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             FC_TICK(11);
             __syncthreads();
@@ -634,11 +662,27 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
         if constexpr (TMA) {
             if (!fk_mbar_wait(bar, phase)) return;
             phase ^= 1u;
+            // Rows ky = 0 and ky = N/2 are real after the column pass, so they travel through
+            // the row pass as one complex row Z = X_0 + i X_{N/2}.  For N <= 32 the whole CTA
+            // forms Z in the staging tile first (one element per thread, one more barrier), so
+            // that the two warps holding the packed rows do no more work than the others.
+            constexpr bool WIDE_COMBINE = (N <= 32);
+            if constexpr (WIDE_COMBINE) {
+                for (int it = tid; it < G * N; it += T) {
+                    const int g = it % G, kx = it / G;
+                    float* a = sStage + (size_t)kx * NC * G + g;
+                    const float x0r = a[0], x0i = a[B * G], xnr = a[M * G], xni = a[(B + M) * G];
+                    a[0] = x0r - xni;
+                    a[B * G] = x0i + xnr;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the next TMA fill
+                __syncthreads();
+            }
             const float* sb = sStage + kyp * G + gB;
             auto load = [&](auto Kx) -> float2 {
                 constexpr int kx = decltype(Kx)::value;
                 float2 v = make_float2(sb[kx * NC * G], sb[(B + kx * NC) * G]);
-                if (packed) {       // row ky = N/2 rides as i times itself
+                if (!WIDE_COMBINE && packed) {       // row ky = N/2 rides as i times itself
                     v.x -= sb[(B + kx * NC + M) * G];
                     v.y += sb[(kx * NC + M) * G];
                 }
