@@ -666,7 +666,7 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             // the row pass as one complex row Z = X_0 + i X_{N/2}.  For N <= 32 the whole CTA
             // forms Z in the staging tile first (one element per thread, one more barrier), so
             // that the two warps holding the packed rows do no more work than the others.
-            constexpr bool WIDE_COMBINE = (N <= 32);
+            constexpr bool WIDE_COMBINE = (N <= 64);
             if constexpr (WIDE_COMBINE) {
                 for (int it = tid; it < G * N; it += T) {
                     const int g = it % G, kx = it / G;
