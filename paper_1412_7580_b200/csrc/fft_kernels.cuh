@@ -759,19 +759,34 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
                 });
                 irfft<N>(Xr, Xi, v);
             }
-            // the crop is the first hc rows: one running pointer, one uniform test per row
+            // the crop is the first hc rows.  One running pointer and one predicated store
+            // per row: written as PTX so that the row test stays a predicate (the compiler
+            // otherwise builds a branch and fresh 64-bit address arithmetic per row)
             float* dst = p.real_out + ((size_t)row * p.C + c0 + gA) * hw + cA;
             const float scale = p.scale;
-            const bool acc = p.accumulate != 0;
-            static_for<N>([&](auto Rr) {
-                constexpr int r = decltype(Rr)::value;
-                if (r < hc) {
-                    float o = v[r] * scale;
-                    if (acc) o += *dst;
-                    *dst = o;
+            if (!p.accumulate && 2 * hc > N) {
+                static_for<N>([&](auto Rr) {
+                    constexpr int r = decltype(Rr)::value;
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\t"
+                        "setp.lt.s32 p, %2, %3;\n\t"
+                        "@p st.global.f32 [%0], %1;\n\t}"
+                        ::"l"(dst), "f"(v[r] * scale), "r"(r), "r"(hc) : "memory");
                     dst += wc;
-                }
-            });
+                });
+            } else {
+                // short crops (filter gradients) and accumulation: a uniform branch per row
+                const bool acc = p.accumulate != 0;
+                static_for<N>([&](auto Rr) {
+                    constexpr int r = decltype(Rr)::value;
+                    if (r < hc) {
+                        float o = v[r] * scale;
+                        if (acc) o += *dst;
+                        *dst = o;
+                        dst += wc;
+                    }
+                });
+            }
         }
     }
 }
