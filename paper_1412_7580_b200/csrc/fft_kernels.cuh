@@ -204,6 +204,11 @@ __device__ __forceinline__ void load_split_narrow(Load&& load, int live, float (
     });
 }
 
+// Measurement builds (never the shipped library; results are wrong or partial):
+//   -DFC_EXP_TIMELINE  cycle counts per phase of the forward tile loop (CTA 0, thread 0);
+//   -DFC_EXP_NOMATH    (fft_core.cuh) the butterflies are skipped: data movement only;
+//   -DFC_EXP_TMAONLY   the TMA-staged kernels only move their tiles (input copy, spectrum
+//                      tile load / store), no shared-memory passes and no arithmetic.
 #ifdef FC_EXP_TIMELINE
 __device__ long long fc_timeline[16];
 #define FC_TICK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { long long t_ = clock64(); fc_timeline[i] += t_ - tl_last; tl_last = t_; } } while (0)
@@ -354,6 +359,20 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             phase ^= 1u;
         }
         FC_TICK(1);
+#ifdef FC_EXP_TMAONLY
+        if (TMA) {
+            if (store_pending && is_storer) fk_bulk_wait_read();
+            __syncthreads();
+            pending = (next < total_tiles) ? stage(second_n, row_n, tcol_n) : false;
+            if (is_storer) {
+                const int b0 = (tid & 31) * D;
+                fk_tma_store_3d(tmS, fk_smem_u32(sStage + (size_t)b0 * G), c0, row, b0);
+                fk_bulk_commit();
+            }
+            store_pending = true;
+            continue;
+        }
+#endif
 
         // 2. column transforms.  Wide planes: thread = (plane gA, column cA), cA < w, one real
         //    FFT of length N each.  Narrow planes (filters): four threads per column, thread
@@ -662,6 +681,11 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
         if constexpr (TMA) {
             if (!fk_mbar_wait(bar, phase)) return;
             phase ^= 1u;
+#ifdef FC_EXP_TMAONLY
+            __syncthreads();
+            if (is_fetcher && tile + (int)gridDim.x < p.num_tiles) fetch_tile(row_n, tcol_n);
+            continue;
+#endif
             // Rows ky = 0 and ky = N/2 are real after the column pass, so they travel through
             // the row pass as one complex row Z = X_0 + i X_{N/2}.  For N <= 32 the whole CTA
             // forms Z in the staging tile first (one element per thread, one more barrier), so
