@@ -57,10 +57,17 @@ def load_peaks():
 # crosses HBM once in the FFT stages; the contraction reads two spectra and
 # writes one).
 # ---------------------------------------------------------------------------
-def pass_model(s, which):
-    B = s.n * (s.n // 2 + 1)
+def pass_model(s, which, tile=0):
+    n = tile or s.n
+    B = n * (n // 2 + 1)
     x_el, w_el, y_el = s.S * s.f * s.h * s.w, s.fp * s.f * s.kh * s.kw, s.S * s.fp * s.oh * s.ow
-    x_pl, w_pl, y_pl = s.S * s.f, s.fp * s.f, s.S * s.fp
+    # windows per plane with spatial tiling (fprop and accGrad tile the output plane, bprop the input)
+    T = 1
+    if tile:
+        dh, dw = n - s.kh + 1, n - s.kw + 1
+        cd = lambda a, b: (a + b - 1) // b
+        T = cd(s.h, dh) * cd(s.w, dw) if which == "bprop" else cd(s.oh, dh) * cd(s.ow, dw)
+    x_pl, w_pl, y_pl = s.S * s.f * T, s.fp * s.f, s.S * s.fp * T
     if which == "fprop":
         a, b, c = (x_el, x_pl), (w_el, w_pl), (y_el, y_pl)
     elif which == "bprop":
@@ -74,7 +81,7 @@ def pass_model(s, which):
         "stage_bytes": stage_bytes,                         # fft A, fft B, contraction, ifft
         "b_fft": stage_bytes[0] + stage_bytes[1] + stage_bytes[3],
         "b_gemm": stage_bytes[2],
-        "gemm_flops": 8.0 * s.S * s.f * s.fp * B,
+        "gemm_flops": 8.0 * s.S * T * s.f * s.fp * B,
         "equiv_flops": 2.0 * s.macs,
     }
 
@@ -220,6 +227,9 @@ def run_ours(args, s):
     x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
     plan = fc.conv_plan(*s.args())
     fc.conv_plan_set_math(plan, math)
+    if args.tile:
+        fc.conv_plan_set_tiling(plan, args.tile)
+    tile = fc.conv_plan_tile_basis(plan)
     ws = fc.conv_plan_alloc_workspace(plan)
     eff = fc.conv_plan_effective_math(plan)
     hx, hw_, hdy = (torch.from_numpy(a).pin_memory() for a in (x, w, dy))
@@ -336,7 +346,7 @@ def run_ours(args, s):
     passes, best = {}, None
     kernel_names = ["r2c_fft_both_operands", None, "bin_contraction", "c2r_ifft"]
     for n in names:
-        m = pass_model(s, n)
+        m = pass_model(s, n, tile)
         t_ms = float(np.median(pass_ms[n]))
         t_roof = max(m["b_fft"] / bw, m["gemm_flops"] / (p_tflops * 1e12))
         t_stage = max((m["b_fft"] + m["b_gemm"]) / bw, m["gemm_flops"] / (p_tflops * 1e12))
@@ -370,7 +380,7 @@ def run_ours(args, s):
     # extra (not the headline, which re-transforms every operand in every pass): the same
     # step with the forward spectra shared between the passes of the step
     reuse = None
-    if not args.no_reuse_line:
+    if not args.no_reuse_line and not tile:
         plan_r = fc.conv_plan(*s.args())
         fc.conv_plan_set_math(plan_r, math)
         fc.conv_plan_set_spectrum_reuse(plan_r, True)
@@ -405,7 +415,8 @@ def run_ours(args, s):
             "scaling": "weak", "vs_baseline": None,
             "dtype": "tf32" if eff == fc.MATH_TF32 else "f32", "data": "synthetic",
             "config": {"workload": s.name, "S": s.S, "f": s.f, "fprime": s.fp, "h": s.h, "w": s.w,
-                       "kh": s.kh, "kw": s.kw, "n": s.n, "passes": "fprop+bprop+accgrad",
+                       "kh": s.kh, "kw": s.kw, "n": s.n, "tile_basis": tile,
+                       "passes": "fprop+bprop+accgrad",
                        "parallelism": "dp%d over S" % world,
                        "l2": "working set %.0f MB > 126 MB L2, no flush" % (
                            (ws.numel() + 4 * (x.size + w.size + dy.size) * 2) / 1e6)},
@@ -432,6 +443,9 @@ def main():
                     help="S,f,fp,h,w,kh,kw,n : a layer shape of your own instead of --config "
                          "(seeded inputs as in the sweep; used for profiling single shapes)")
     ap.add_argument("--math", default="auto", choices=["auto", "fp32", "tf32"])
+    ap.add_argument("--tile", type=int, default=0,
+                    help="spatial tiling with this basis (8, 16, 32 or 64; 0 = off); bytes, flops and the "
+                         "roofline in the output are then those of the tiled method")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-reuse-line", action="store_true",

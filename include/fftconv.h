@@ -143,9 +143,31 @@ int conv_accgrad(conv_plan_t* plan, const float* dy, const float* x, float* dw, 
  * modified since that spectrum was computed, and the passes must be ordered on
  * one stream (or synchronised by the caller); otherwise call
  * conv_plan_invalidate_spectra first.  Changing the setting or the workspace
- * invalidates everything.  Results are identical to the non-reusing passes. */
+ * invalidates everything.  Results are identical to the non-reusing passes.
+ * EUNSUPPORTED together with spatial tiling (the passes then use different windows). */
 int conv_plan_set_spectrum_reuse(conv_plan_t* plan, int enable);
 int conv_plan_invalidate_spectra(conv_plan_t* plan);
+
+/* Spatial tiling (Section 6): with n_tile in {8, 16, 32, 64} smaller than the plan's basis n,
+ * every pass decomposes its planes into tiles that fit an n_tile x n_tile basis instead of
+ * padding kernels and planes to n x n.  With steps dh = n_tile - kh + 1, dw = n_tile - kw + 1:
+ *   fprop  : each dh x dw tile of y is the valid cross-correlation of the n_tile x n_tile window
+ *            of x at the same origin with w (the paper's y[i, i+d] = x[i, i+d+w] (star) c);
+ *   bprop  : each dh x dw tile of dx is the full convolution of w with the n_tile x n_tile window
+ *            of dy that starts kh-1 rows and kw-1 columns before the tile (zero outside dy);
+ *   accGrad: dw is the sum over the minibatch AND over the tiles of (dh x dw tile of dy)
+ *            (star) (n_tile x n_tile window of x), the paper's tiled sum for the kernel gradient.
+ * The window index joins the minibatch index in the per-bin contraction (S T rows instead of S,
+ * T = tiles per plane), the weight spectra shrink from n(n/2+1) to n_tile(n_tile/2+1) bins, and
+ * windows are read with clipped loads and written straight into the planes: nothing is
+ * gathered or padded in memory.  Results are those of the untiled passes up to rounding.
+ * n_tile == 0 (or == n) switches tiling off.  Changes the workspace size: query it again and
+ * lend a workspace of that size.  EUNSUPPORTED: n_tile not in {8,16,32,64}, spectrum reuse
+ * enabled, or more than 2^30 windows; EINVAL: n_tile > n or n_tile < max(kh, kw). */
+int conv_plan_set_tiling(conv_plan_t* plan, int n_tile);
+
+/* The tile basis in use, 0 when tiling is off. */
+int conv_plan_tile_basis(const conv_plan_t* plan);
 
 /* Reads the plan's device status word (synchronises the device).  FFTCONV_OK,
  * or FFTCONV_EDEVICE_TIMEOUT if a bounded wait inside a kernel gave up since

@@ -20,6 +20,7 @@ EXPORTS = (
     "conv_plan", "conv_plan_set_math", "conv_plan_effective_math", "conv_plan_pass_math",
     "conv_plan_workspace_bytes",
     "conv_plan_set_workspace", "conv_plan_set_spectrum_reuse", "conv_plan_invalidate_spectra",
+    "conv_plan_set_tiling", "conv_plan_tile_basis",
     "conv_fprop", "conv_fprop_noalloc", "conv_bprop", "conv_accgrad", "conv_plan_status",
     "conv_plan_destroy", "conv_plan_enable_stage_timing", "conv_plan_stage_times_ms", "fft2d_r2c", "fft2d_c2r", "fftconv_bin_contract",
     "fftconv_status_string", "fftconv_launch_count",
@@ -53,6 +54,8 @@ def lib():
         L.conv_plan_set_workspace.argtypes = [p, p, z]
         L.conv_plan_set_spectrum_reuse.argtypes = [p, i]
         L.conv_plan_invalidate_spectra.argtypes = [p]
+        L.conv_plan_set_tiling.argtypes = [p, i]
+        L.conv_plan_tile_basis.argtypes = [p]
         L.conv_fprop.argtypes = [p, p, p, p, p]
         L.conv_fprop_noalloc.argtypes = [p, p, p, p, p]
         L.conv_bprop.argtypes = [p, p, p, p, p]
@@ -171,6 +174,17 @@ def conv_plan_set_spectrum_reuse(plan: Plan, enable=True) -> None:
     workspace size: size and lend the workspace after this call)."""
     _check(lib().conv_plan_set_spectrum_reuse(plan.handle, int(bool(enable))),
            "conv_plan_set_spectrum_reuse")
+
+
+def conv_plan_set_tiling(plan: Plan, n_tile: int) -> None:
+    """Spatial tiling with an n_tile x n_tile basis (0 = off); changes the workspace size:
+    size and lend the workspace after this call."""
+    _check(lib().conv_plan_set_tiling(plan.handle, int(n_tile)), "conv_plan_set_tiling")
+    plan.workspace = None
+
+
+def conv_plan_tile_basis(plan: Plan) -> int:
+    return lib().conv_plan_tile_basis(plan.handle)
 
 
 def conv_plan_invalidate_spectra(plan: Plan) -> None:

@@ -67,6 +67,16 @@ struct FftParams {
     int in_bytes;           // shared-memory bytes reserved for the real tile (multiple of 128)
     float scale;            // inverse
     int accumulate;         // inverse
+    // Spatial tiling (Section 6): win != 0 makes every matrix row (s, ty, tx) a window of plane s
+    // of a larger H x W plane instead of a whole plane.  Tiles step by (step_y, step_x).
+    // Forward: the window of h x w samples starts at (ty step_y + oy, tx step_x + ox), samples
+    // outside the plane read as zero.  Inverse: rows [oy, oy + h) and columns [ox, ox + w) of the
+    // transform's output go to the plane at (ty step_y, tx step_x), clipped at the plane's edge.
+    int win;
+    int H, W;
+    int nty, ntx;
+    int step_y, step_x;
+    int oy, ox;
 };
 
 // Geometry of the half-spectrum scratch ("mid") of one plane in shared memory:
@@ -301,12 +311,43 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
 
     // Stage the planes of a tile.  Returns true if the copy is asynchronous (wait on the
     // barrier before reading), false if it was done with plain loads by all threads.
+    bool win_pending = false;       // windowed tile on its way in through cp.async
     auto stage = [&](bool second, int row, int tcol) -> bool {
         const int sh = second ? p1.h : p0.h, sw = second ? p1.w : p0.w;
         const int sC = second ? p1.C : p0.C;
         const float* base = second ? p1.real_in : p0.real_in;
         const int c0 = tcol * G;
         const int gcount = min(G, sC - c0);
+        if (second ? p1.win : p0.win) {
+            // window of a larger plane: clipped loads (Section 5.1), one plane row per N lanes
+            const FftParams& pw = second ? p1 : p0;
+            const int nt = pw.nty * pw.ntx;
+            const int s = row / nt, t = row - s * nt;
+            const int ty = t / pw.ntx, tx = t - ty * pw.ntx;
+            const int y0 = ty * pw.step_y + pw.oy, x0 = tx * pw.step_x + pw.ox;
+            const int rr = tid / N, cc = tid - rr * N;
+            const int xx = x0 + cc;
+            const bool col_ok = (cc < sw) && xx >= 0 && xx < pw.W;
+            // 4-byte asynchronous copies; a sample outside the plane is a copy of zero bytes,
+            // which writes a zero.  Completion: every thread waits for its own copies, then a
+            // barrier (win_pending, at the top of the tile loop).
+            if (cc < sw) {
+                for (int g = 0; g < gcount; ++g) {
+                    const float* pl0 = base + ((size_t)s * sC + c0 + g) * ((size_t)pw.H * pw.W);
+                    const uint32_t dstp = fk_smem_u32(sIn + g * sh * sw + cc);
+                    for (int r = rr; r < sh; r += G) {
+                        const int yy = y0 + r;
+                        const bool ok = col_ok && yy >= 0 && yy < pw.H;
+                        const float* src = ok ? pl0 + (size_t)yy * pw.W + xx : pl0;
+                        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;"
+                                     ::"r"(dstp + 4u * (uint32_t)(r * sw)), "l"(src), "r"(ok ? 4 : 0)
+                                     : "memory");
+                    }
+                }
+            }
+            win_pending = true;
+            return false;
+        }
         const float* src = base + ((size_t)row * sC + c0) * (sh * sw);
         const int total = gcount * sh * sw;
         if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
@@ -357,6 +398,11 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
         if (pending) {
             if (!fk_mbar_wait(bar, phase)) return;     // copy never landed: give up
             phase ^= 1u;
+        }
+        if (win_pending) {
+            asm volatile("cp.async.wait_all;" ::: "memory");
+            __syncthreads();
+            win_pending = false;
         }
         FC_TICK(1);
 #ifdef FC_EXP_TMAONLY
@@ -767,7 +813,18 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
 
         // 2. column transforms: thread = (plane gA, column cA), cA < wc; results go straight
         //    to global memory (lanes run along the row of the plane: contiguous segments)
-        if (gA < gcount && cA < wc) {
+        int win_hc = hc, win_wc = wc;
+        size_t win_base = 0;
+        if (p.win) {
+            const int nt = p.nty * p.ntx;
+            const int s = row / nt, t = row - s * nt;
+            const int ty = t / p.ntx, tx = t - ty * p.ntx;
+            win_hc = min(hc, p.H - ty * p.step_y);
+            win_wc = min(wc, p.W - tx * p.step_x);
+            win_base = ((size_t)s * p.C + c0 + gA) * ((size_t)p.H * p.W) +
+                       (size_t)(ty * p.step_y) * p.W + tx * p.step_x;
+        }
+        if (gA < gcount && (p.win ? (cA >= p.ox && cA < p.ox + win_wc) : (cA < wc))) {
             float v[N];
             {
                 float Xr[NC], Xi[NC];
@@ -788,7 +845,21 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             // otherwise builds a branch and fresh 64-bit address arithmetic per row)
             float* dst = p.real_out + ((size_t)row * p.C + c0 + gA) * hw + cA;
             const float scale = p.scale;
-            if (!p.accumulate && 2 * hc > N) {
+            if (p.win) {
+                // rows [oy, oy + win_hc) of the transform go to the tile's place in the plane
+                dst = p.real_out + win_base + (cA - p.ox);
+                const bool acc = p.accumulate != 0;
+                const int r0 = p.oy, r1 = p.oy + win_hc, pitch = p.W;
+                static_for<N>([&](auto Rr) {
+                    constexpr int r = decltype(Rr)::value;
+                    if (r >= r0 && r < r1) {
+                        float o = v[r] * scale;
+                        if (acc) o += *dst;
+                        *dst = o;
+                        dst += pitch;
+                    }
+                });
+            } else if (!p.accumulate && 2 * hc > N) {
                 static_for<N>([&](auto Rr) {
                     constexpr int r = decltype(Rr)::value;
                     asm volatile(

@@ -40,6 +40,8 @@ struct OperandDesc {
     SpecDesc spec;
     int h, w;               // plane size (forward) or crop window (inverse)
     int kind;               // which tensor family: 0 = x / dx, 1 = w / dw, 2 = y / dy
+    // spatial tiling: the operand's matrix rows are windows (s, ty, tx) of H x W planes
+    int win, H, W, nty, ntx, step_y, step_x, oy, ox;
 };
 
 struct PassDesc {
@@ -55,6 +57,7 @@ enum { PASS_FPROP = 0, PASS_BPROP = 1, PASS_ACCGRAD = 2 };
 struct conv_plan_s {
     int S, f, fp, h, w, kh, kw, n;
     int oh, ow, bins;
+    int n_full;        // the basis given to conv_plan; n is the one in use (the tile's when tiling)
     int math;          // requested fftconv_math
     void* ws;
     size_t ws_bytes;
@@ -76,12 +79,63 @@ namespace {
 //   fprop  : Y^[b][s][j]  = sum_i X^[b][s][i]        conj W^[b][j][i]
 //   bprop  : dX^[b][s][i] = sum_j dY^[b][s][j]       W^[b][j][i]        (B read as [k=j][i])
 //   accGrad: dW^[b][j][i] = sum_s conj dY^[b][s][j]  X^[b][s][i]        (A as [k=s][j], B as [k=s][i])
-PassDesc describe(const conv_plan_s& p, int pass) {
+// Spatial tiling (Section 6): with a tile basis n < the plane, every pass works on windows.
+// Steps dh = n - kh + 1, dw = n - kw + 1.
+//   fprop  : y tile (ty, tx) of dh x dw       = x window of n x n at the same origin (star) w
+//   bprop  : dx tile of dh x dw at (ty dh, ..) = rows kh-1.. of (dy window of n x n starting
+//            kh-1 rows and kw-1 columns before the tile's origin, zero outside the plane) * w
+//   accGrad: dw = sum over s and tiles of  dy tile of dh x dw (star) x window of n x n
+// The window index joins the minibatch index: matrix rows (s, ty, tx), S T of them; accGrad
+// sums over them.  fprop and accGrad tile the output plane, bprop tiles the input plane.
+PassDesc describe_tiled(const conv_plan_s& p, int pass) {
     PassDesc d{};
     auto spec = [](int R, int C) { return SpecDesc{R, C, round4(C)}; };
-    const OperandDesc X = {spec(p.S, p.f), p.h, p.w, 0};
-    const OperandDesc W = {spec(p.fp, p.f), p.kh, p.kw, 1};
-    const OperandDesc Y = {spec(p.S, p.fp), p.oh, p.ow, 2};
+    const int n = p.n, dh = n - p.kh + 1, dw = n - p.kw + 1;
+    auto cdiv = [](int a, int b) { return (a + b - 1) / b; };
+    const int oty = cdiv(p.oh, dh), otx = cdiv(p.ow, dw);       // tiles of the output plane
+    const int ity = cdiv(p.h, dh), itx = cdiv(p.w, dw);         // tiles of the input plane
+    auto mn = [](int a, int b) { return a < b ? a : b; };
+    const OperandDesc W = {spec(p.fp, p.f), p.kh, p.kw, 1, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    switch (pass) {
+        case PASS_FPROP: {
+            const int T = oty * otx;
+            d.a = {spec(p.S * T, p.f), mn(n, p.h), mn(n, p.w), 0, 1, p.h, p.w, oty, otx, dh, dw, 0, 0};
+            d.b = W;
+            d.c = {spec(p.S * T, p.fp), mn(dh, p.oh), mn(dw, p.ow), 2, 1, p.oh, p.ow, oty, otx, dh, dw, 0, 0};
+            d.M = p.S * T; d.N = p.fp; d.K = p.f;
+            d.transA = 0; d.transB = 0; d.conjA = 0; d.conjB = 1;
+            break;
+        }
+        case PASS_BPROP: {
+            const int T = ity * itx;
+            d.a = {spec(p.S * T, p.fp), n, n, 2, 1, p.oh, p.ow, ity, itx, dh, dw, -(p.kh - 1), -(p.kw - 1)};
+            d.b = W;
+            d.c = {spec(p.S * T, p.f), mn(dh, p.h), mn(dw, p.w), 0, 1, p.h, p.w, ity, itx, dh, dw,
+                   p.kh - 1, p.kw - 1};
+            d.M = p.S * T; d.N = p.f; d.K = p.fp;
+            d.transA = 0; d.transB = 1; d.conjA = 0; d.conjB = 0;
+            break;
+        }
+        default: {
+            const int T = oty * otx;
+            d.a = {spec(p.S * T, p.fp), mn(dh, p.oh), mn(dw, p.ow), 2, 1, p.oh, p.ow, oty, otx, dh, dw, 0, 0};
+            d.b = {spec(p.S * T, p.f), mn(n, p.h), mn(n, p.w), 0, 1, p.h, p.w, oty, otx, dh, dw, 0, 0};
+            d.c = W;
+            d.M = p.fp; d.N = p.f; d.K = p.S * T;
+            d.transA = 1; d.transB = 1; d.conjA = 1; d.conjB = 0;
+            break;
+        }
+    }
+    return d;
+}
+
+PassDesc describe(const conv_plan_s& p, int pass) {
+    if (p.n != p.n_full) return describe_tiled(p, pass);
+    PassDesc d{};
+    auto spec = [](int R, int C) { return SpecDesc{R, C, round4(C)}; };
+    const OperandDesc X = {spec(p.S, p.f), p.h, p.w, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    const OperandDesc W = {spec(p.fp, p.f), p.kh, p.kw, 1, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+    const OperandDesc Y = {spec(p.S, p.fp), p.oh, p.ow, 2, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     switch (pass) {
         case PASS_FPROP:
             d.a = X; d.b = W; d.c = Y;
@@ -177,14 +231,17 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         fp.real_in = in; fp.spec_out = spec;
         fp.h = o.h; fp.w = o.w;
         fp.R = o.spec.R; fp.C = o.spec.C; fp.ld = o.spec.ld;
+        fp.win = o.win; fp.H = o.H; fp.W = o.W; fp.nty = o.nty; fp.ntx = o.ntx;
+        fp.step_y = o.step_y; fp.step_x = o.step_x; fp.oy = o.oy; fp.ox = o.ox;
         return fp;
     };
     const bool timing = plan->timing && plan->ev_made;
     auto mark = [&](int i) { if (timing) cudaEventRecord(plan->ev[i], st); };
     // large planes run the two-pass transforms (one launch per operand, scratch behind the spectra)
-    const bool big = fc::big_uses_two_pass(plan->n);
+    const bool tiled = plan->n != plan->n_full;
+    const bool big = !tiled && fc::big_uses_two_pass(plan->n);
     float* scratch = reinterpret_cast<float*>(base + align_up(spectra_bytes(plan), kAlign));
-    const size_t scratch_bytes = fc::big_scratch_bytes(plan->n);
+    const size_t scratch_bytes = tiled ? 0 : fc::big_scratch_bytes(plan->n);
     auto forward = [&](const fc::FftParams& pa, const fc::FftParams* pb) -> cudaError_t {
         g_launches.fetch_add((big && pb) ? 2 : 1, std::memory_order_relaxed);
         if (!big) return fc::launch_r2c<true>(plan->n, pa, pb, st);
@@ -228,6 +285,8 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     ip.spec_in = specC; ip.real_out = c_out;
     ip.h = d.c.h; ip.w = d.c.w;
     ip.R = d.c.spec.R; ip.C = d.c.spec.C; ip.ld = d.c.spec.ld;
+    ip.win = d.c.win; ip.H = d.c.H; ip.W = d.c.W; ip.nty = d.c.nty; ip.ntx = d.c.ntx;
+    ip.step_y = d.c.step_y; ip.step_x = d.c.step_x; ip.oy = d.c.oy; ip.ox = d.c.ox;
     ip.scale = 1.0f / ((float)plan->n * (float)plan->n);
     ip.accumulate = accumulate ? 1 : 0;
     g_launches.fetch_add(1, std::memory_order_relaxed);
@@ -258,6 +317,7 @@ FFTCONV_API int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, in
     conv_plan_s* p = new (std::nothrow) conv_plan_s();
     if (!p) return FFTCONV_EINVAL;
     p->S = S; p->f = f; p->fp = fprime; p->h = h; p->w = w; p->kh = kh; p->kw = kw; p->n = n;
+    p->n_full = n;
     p->oh = h - kh + 1; p->ow = w - kw + 1;
     p->bins = n * (n / 2 + 1);
     p->math = FFTCONV_MATH_AUTO;
@@ -291,7 +351,34 @@ FFTCONV_API int conv_plan_pass_math(const conv_plan_t* plan, int pass) {
 
 FFTCONV_API size_t conv_plan_workspace_bytes(const conv_plan_t* plan) {
     if (!plan) return 0;
-    return align_up(spectra_bytes(plan), kAlign) + fc::big_scratch_bytes(plan->n);
+    return align_up(spectra_bytes(plan), kAlign) +
+           (plan->n != plan->n_full ? 0 : fc::big_scratch_bytes(plan->n));
+}
+
+FFTCONV_API int conv_plan_set_tiling(conv_plan_t* plan, int n_tile) {
+    if (!plan) return FFTCONV_EINVAL;
+    if (n_tile == 0 || n_tile == plan->n_full) {
+        plan->n = plan->n_full;
+    } else {
+        // one-pass transforms only; a tile must produce at least one output sample per axis
+        if (n_tile != 8 && n_tile != 16 && n_tile != 32 && n_tile != 64) return FFTCONV_EUNSUPPORTED;
+        if (n_tile > plan->n_full) return FFTCONV_EINVAL;
+        if (n_tile < plan->kh || n_tile < plan->kw) return FFTCONV_EINVAL;
+        if (plan->reuse) return FFTCONV_EUNSUPPORTED;
+        const long long dh = n_tile - plan->kh + 1, dw = n_tile - plan->kw + 1;
+        const long long T = ((plan->h + dh - 1) / dh) * ((plan->w + dw - 1) / dw);
+        const long long pmax = plan->f > plan->fp ? plan->f : plan->fp;
+        if ((long long)plan->S * T * pmax > (1LL << 30)) return FFTCONV_EUNSUPPORTED;
+        plan->n = n_tile;
+    }
+    plan->bins = plan->n * (plan->n / 2 + 1);
+    plan->cached[0] = plan->cached[1] = plan->cached[2] = nullptr;
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_plan_tile_basis(const conv_plan_t* plan) {
+    if (!plan) return FFTCONV_EINVAL;
+    return plan->n != plan->n_full ? plan->n : 0;
 }
 
 FFTCONV_API int conv_plan_set_workspace(conv_plan_t* plan, void* dev_ptr, size_t bytes) {
@@ -308,6 +395,7 @@ FFTCONV_API int conv_plan_set_workspace(conv_plan_t* plan, void* dev_ptr, size_t
 
 FFTCONV_API int conv_plan_set_spectrum_reuse(conv_plan_t* plan, int enable) {
     if (!plan) return FFTCONV_EINVAL;
+    if (enable && plan->n != plan->n_full) return FFTCONV_EUNSUPPORTED;   // not with tiling
     plan->reuse = enable ? 1 : 0;
     plan->cached[0] = plan->cached[1] = plan->cached[2] = nullptr;
     return FFTCONV_OK;

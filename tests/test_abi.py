@@ -97,3 +97,26 @@ def test_calls_without_workspace_or_pointers_fail_cleanly(L):
     assert L.fft2d_c2r(one, one, 1, 8, 9, 8, 1.0, 0, z) == b.EINVAL
     assert b.status_string(b.EWORKSPACE).startswith("workspace")
     b.conv_plan_destroy(p)
+
+
+def test_tiling_argument_checks(L):
+    import paper_1412_7580_b200 as fc
+    p = fc.conv_plan(2, 3, 4, 31, 31, 9, 9, 32)
+    with pytest.raises(fc.FftConvError) as e:
+        fc.conv_plan_set_tiling(p, 12)                 # not a supported basis
+    assert e.value.status == fc.binding.EUNSUPPORTED
+    with pytest.raises(fc.FftConvError) as e:
+        fc.conv_plan_set_tiling(p, 8)                  # smaller than the kernel
+    assert e.value.status == fc.binding.EINVAL
+    with pytest.raises(fc.FftConvError) as e:
+        fc.conv_plan_set_tiling(p, 64)                 # larger than the plan's basis
+    assert e.value.status == fc.binding.EINVAL
+    before = fc.conv_plan_workspace_bytes(p)
+    fc.conv_plan_set_tiling(p, 16)
+    assert fc.conv_plan_tile_basis(p) == 16 and fc.conv_plan_workspace_bytes(p) != before
+    with pytest.raises(fc.FftConvError) as e:
+        fc.conv_plan_set_spectrum_reuse(p, True)       # the passes use different windows
+    assert e.value.status == fc.binding.EUNSUPPORTED
+    fc.conv_plan_set_tiling(p, 0)
+    assert fc.conv_plan_tile_basis(p) == 0 and fc.conv_plan_workspace_bytes(p) == before
+    fc.conv_plan_destroy(p)
