@@ -231,7 +231,7 @@ __device__ long long fc_timeline[16];
 // ALIAS: the half-spectrum scratch overwrites the staging area of the real tile
 // (no prefetch of the next tile); used where one tile nearly fills shared memory.
 // ---------------------------------------------------------------------------
-template <int N, int G, int LAYOUT, bool ALIAS, bool SALIAS, int MINB>
+template <int N, int G, int LAYOUT, bool ALIAS, bool SALIAS, int MINB, bool WIN = false>
 __global__ void __launch_bounds__(N* G, MINB)
 r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUtensorMap tmS1,
            const FftParams p0, const FftParams p1) {
@@ -318,7 +318,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
         const float* base = second ? p1.real_in : p0.real_in;
         const int c0 = tcol * G;
         const int gcount = min(G, sC - c0);
-        if (second ? p1.win : p0.win) {
+        if (WIN && (second ? p1.win : p0.win)) {
             // window of a larger plane: clipped loads (Section 5.1), one plane row per N lanes
             const FftParams& pw = second ? p1 : p0;
             const int nt = pw.nty * pw.ntx;
@@ -399,7 +399,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             if (!fk_mbar_wait(bar, phase)) return;     // copy never landed: give up
             phase ^= 1u;
         }
-        if (win_pending) {
+        if (WIN && win_pending) {
             asm volatile("cp.async.wait_all;" ::: "memory");
             __syncthreads();
             win_pending = false;
@@ -667,7 +667,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
 // ---------------------------------------------------------------------------
 // Inverse: half spectra -> cropped, scaled real planes.
 // ---------------------------------------------------------------------------
-template <int N, int G, int LAYOUT, int MINB>
+template <int N, int G, int LAYOUT, int MINB, bool WIN = false>
 __global__ void __launch_bounds__(N* G, MINB)
 c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
     constexpr int T = N * G, NC = N / 2 + 1, M = N / 2, HALF = T / 2, B = N * NC;
@@ -815,7 +815,7 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
         //    to global memory (lanes run along the row of the plane: contiguous segments)
         int win_hc = hc, win_wc = wc;
         size_t win_base = 0;
-        if (p.win) {
+        if (WIN && p.win) {
             const int nt = p.nty * p.ntx;
             const int s = row / nt, t = row - s * nt;
             const int ty = t / p.ntx, tx = t - ty * p.ntx;
@@ -824,7 +824,7 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             win_base = ((size_t)s * p.C + c0 + gA) * ((size_t)p.H * p.W) +
                        (size_t)(ty * p.step_y) * p.W + tx * p.step_x;
         }
-        if (gA < gcount && (p.win ? (cA >= p.ox && cA < p.ox + win_wc) : (cA < wc))) {
+        if (gA < gcount && ((WIN && p.win) ? (cA >= p.ox && cA < p.ox + win_wc) : (cA < wc))) {
             float v[N];
             {
                 float Xr[NC], Xi[NC];
@@ -845,7 +845,7 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             // otherwise builds a branch and fresh 64-bit address arithmetic per row)
             float* dst = p.real_out + ((size_t)row * p.C + c0 + gA) * hw + cA;
             const float scale = p.scale;
-            if (p.win) {
+            if (WIN && p.win) {
                 // rows [oy, oy + win_hc) of the transform go to the tile's place in the plane
                 dst = p.real_out + win_base + (cA - p.ox);
                 const bool acc = p.accumulate != 0;
@@ -995,7 +995,12 @@ static cudaError_t launch_r2c_n(FftParams pa, const FftParams* pb_in, cudaStream
         if (!make_spec_map<N, G>(&tma, pa.spec_out, pa)) return cudaErrorInvalidValue;
         if (pb_in && !make_spec_map<N, G>(&tmb, pb.spec_out, pb)) return cudaErrorInvalidValue;
     }
-    auto kern = r2c_kernel<N, G, LAYOUT, Cfg::ALIAS, SALIAS, Cfg::MINB>;
+    // the windowed variant (spatial tiling) is a separate instantiation, so that the plain
+    // kernels carry none of its code
+    const bool win = pa.win || (pb_in && pb.win);
+    auto kern = (win && LAYOUT == LAYOUT_FREQ_TMA) ? r2c_kernel<N, G, LAYOUT, Cfg::ALIAS, SALIAS, Cfg::MINB, LAYOUT == LAYOUT_FREQ_TMA>
+                                                   : r2c_kernel<N, G, LAYOUT, Cfg::ALIAS, SALIAS, Cfg::MINB, false>;
+    if (win && LAYOUT != LAYOUT_FREQ_TMA) return cudaErrorInvalidValue;
     int grid = 0;
     cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), N * G, smem,
                                     (long long)pa.num_tiles + pb.num_tiles, &grid);
@@ -1018,7 +1023,9 @@ static cudaError_t launch_c2r_n(FftParams p, cudaStream_t st) {
         smem += (size_t)2 * N * (N / 2 + 1) * G * sizeof(float);
         if (!make_spec_map<N, G>(&tm, p.spec_in, p)) return cudaErrorInvalidValue;
     }
-    auto kern = c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV>;
+    if (p.win && LAYOUT != LAYOUT_FREQ_TMA) return cudaErrorInvalidValue;
+    auto kern = (p.win && LAYOUT == LAYOUT_FREQ_TMA) ? c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV, LAYOUT == LAYOUT_FREQ_TMA>
+                                                     : c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV, false>;
     int grid = 0;
     cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), N * G, smem, p.num_tiles, &grid);
     if (e != cudaSuccess) return e;
