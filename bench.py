@@ -34,9 +34,34 @@ FP32_FFMA_TFLOPS_NOMINAL = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x lanes x 2 fl
 # DRAM bytes (read + write) of one launch from the ncu captures summarised under profiles/,
 # keyed by (workload, kernel, pass); None where no capture exists.
 NCU_TRAFFIC = {
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "bprop"): 291.9e6,
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "accgrad"): 287.4e6,
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "fprop"): 157.2e6,
+    # (workload, kernel, pass): read + write, profiles/dram_traffic_per_launch_three_layer_configs.md
+    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "fprop"): 156.5e6,
+    ("mid_S128_f96_fp256_31x31_k5", "bin_contraction", "fprop"): 242.4e6,
+    ("mid_S128_f96_fp256_31x31_k5", "c2r_ifft", "fprop"): 193.9e6,
+    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "bprop"): 291.0e6,
+    ("mid_S128_f96_fp256_31x31_k5", "bin_contraction", "bprop"): 277.1e6,
+    ("mid_S128_f96_fp256_31x31_k5", "c2r_ifft", "bprop"): 54.4e6,
+    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "accgrad"): 286.9e6,
+    ("mid_S128_f96_fp256_31x31_k5", "bin_contraction", "accgrad"): 257.7e6,
+    ("mid_S128_f96_fp256_31x31_k5", "c2r_ifft", "accgrad"): 107.6e6,
+    ("largek_S128_f64_fp64_64x64_k11", "r2c_fft_both_operands", "fprop"): 293.1e6,
+    ("largek_S128_f64_fp64_64x64_k11", "bin_contraction", "fprop"): 290.4e6,
+    ("largek_S128_f64_fp64_64x64_k11", "c2r_ifft", "fprop"): 192.0e6,
+    ("largek_S128_f64_fp64_64x64_k11", "r2c_fft_both_operands", "bprop"): 251.9e6,
+    ("largek_S128_f64_fp64_64x64_k11", "bin_contraction", "bprop"): 290.1e6,
+    ("largek_S128_f64_fp64_64x64_k11", "c2r_ifft", "bprop"): 222.4e6,
+    ("largek_S128_f64_fp64_64x64_k11", "r2c_fft_both_operands", "accgrad"): 454.2e6,
+    ("largek_S128_f64_fp64_64x64_k11", "bin_contraction", "accgrad"): 324.1e6,
+    ("largek_S128_f64_fp64_64x64_k11", "c2r_ifft", "accgrad"): 69.3e6,
+    ("deep_S128_f384_fp384_13x13_k3", "r2c_fft_both_operands", "fprop"): 210.8e6,
+    ("deep_S128_f384_fp384_13x13_k3", "bin_contraction", "fprop"): 251.7e6,
+    ("deep_S128_f384_fp384_13x13_k3", "c2r_ifft", "fprop"): 56.8e6,
+    ("deep_S128_f384_fp384_13x13_k3", "r2c_fft_both_operands", "bprop"): 198.2e6,
+    ("deep_S128_f384_fp384_13x13_k3", "bin_contraction", "bprop"): 251.8e6,
+    ("deep_S128_f384_fp384_13x13_k3", "c2r_ifft", "bprop"): 57.1e6,
+    ("deep_S128_f384_fp384_13x13_k3", "r2c_fft_both_operands", "accgrad"): 114.6e6,
+    ("deep_S128_f384_fp384_13x13_k3", "bin_contraction", "accgrad"): 222.3e6,
+    ("deep_S128_f384_fp384_13x13_k3", "c2r_ifft", "accgrad"): 172.6e6,
 }
 
 
