@@ -397,7 +397,7 @@ def run_ours(args, s):
         ach = bbytes / (dur_ms * 1e-3) / 1e9
         roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": ach / peaks["hbm_gbs"]}
-    roof.update({"traffic": NCU_TRAFFIC.get((s.name, kernel_names[bk], bn)),
+    roof.update({"traffic": None if tile else NCU_TRAFFIC.get((s.name, kernel_names[bk], bn)),
                  "kernel": "%s/%s" % (bn, kernel_names[bk]),
                  "kernel_ms": dur_ms, "algorithmic_bytes": bbytes,
                  "peak_source": peaks["source"] + (" sustained bf16 / 2" if roof["bound"] == "tensor" else "")})
