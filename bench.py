@@ -253,7 +253,7 @@ def run_ours(args, s):
     plan = fc.conv_plan(*s.args())
     fc.conv_plan_set_math(plan, math)
     if args.tile:
-        fc.conv_plan_set_tiling(plan, args.tile)
+        fc.conv_plan_set_tiling(plan, args.tile)      # -1: the plan chooses
     tile = fc.conv_plan_tile_basis(plan)
     ws = fc.conv_plan_alloc_workspace(plan)
     eff = fc.conv_plan_effective_math(plan)

@@ -163,7 +163,12 @@ int conv_plan_invalidate_spectra(conv_plan_t* plan);
  * gathered or padded in memory.  Results are those of the untiled passes up to rounding.
  * n_tile == 0 (or == n) switches tiling off.  Changes the workspace size: query it again and
  * lend a workspace of that size.  EUNSUPPORTED: n_tile not in {8,16,32,64}, spectrum reuse
- * enabled, or more than 2^30 windows; EINVAL: n_tile > n or n_tile < max(kh, kw). */
+ * enabled, or more than 2^30 windows; EINVAL: n_tile > n or n_tile < max(kh, kw).
+ * n_tile == FFTCONV_TILE_AUTO lets the plan choose: it estimates a training step for every
+ * admissible basis from the bytes each kernel moves (Section 3.4's one strategy per problem size,
+ * decided by a static model instead of trial runs) and keeps tiling off unless a tile basis is
+ * estimated at least 10 % faster. */
+#define FFTCONV_TILE_AUTO (-1)
 int conv_plan_set_tiling(conv_plan_t* plan, int n_tile);
 
 /* The tile basis in use, 0 when tiling is off. */

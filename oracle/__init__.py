@@ -13,6 +13,8 @@ Functions (paper notation: S, f, fp = f', h, w, kh, kw, n):
   *_at(..., coords)      -> the same elements at sampled coordinates
   dft2d_r2c(x, n)        -> complex128 [batch, n, n/2+1]  (Supplement 8.2)
   idft2d_c2r(X, n, oh, ow, scale) -> float64 [batch, oh, ow]
+  dft1d_r2c(x, n)        -> complex128 [batch, n/2+1]     (Supplement 8.2)
+  idft1d_c2r(X, n, olen, scale)   -> float64 [batch, olen]
   bin_contract(A, B, conjA, conjB) -> complex128 [bins, M, N] (Table 1, Cgemm)
 """
 from __future__ import annotations
@@ -57,6 +59,8 @@ def _load():
             getattr(lib, name).argtypes = [p, p, p, l, p] + [i] * 7
         lib.oracle_dft2d_r2c.argtypes = [p, p, l, i, i, i]
         lib.oracle_idft2d_c2r.argtypes = [p, p, l, i, i, i, d]
+        lib.oracle_dft1d_r2c.argtypes = [p, p, l, i, i]
+        lib.oracle_idft1d_c2r.argtypes = [p, p, l, i, i, d]
         lib.oracle_bin_contract.argtypes = [p, p, p, l, i, i, i, i, i]
         for name in ("oracle_fprop", "oracle_bprop", "oracle_accgrad",
                      "oracle_fprop_at", "oracle_bprop_at", "oracle_accgrad_at",
@@ -165,6 +169,24 @@ def idft2d_c2r(X, n, oh, ow, scale):
     assert X.shape[1:] == (n, n // 2 + 1)
     out = np.empty((batch, oh, ow), dtype=np.float64)
     _load().oracle_idft2d_c2r(_ptr(X), _ptr(out), batch, n, oh, ow, float(scale))
+    return out
+
+
+def dft1d_r2c(x, n):
+    x = _f32(x)
+    batch, ln = x.shape
+    assert n >= ln
+    out = np.empty((batch, n // 2 + 1), dtype=np.complex128)
+    _load().oracle_dft1d_r2c(_ptr(x), _ptr(out), batch, ln, n)
+    return out
+
+
+def idft1d_c2r(X, n, olen, scale):
+    X = np.ascontiguousarray(X, dtype=np.complex128)
+    batch = X.shape[0]
+    assert X.shape[1:] == (n // 2 + 1,)
+    out = np.empty((batch, olen), dtype=np.float64)
+    _load().oracle_idft1d_c2r(_ptr(X), _ptr(out), batch, n, olen, float(scale))
     return out
 
 

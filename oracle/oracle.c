@@ -249,6 +249,58 @@ API void oracle_idft2d_c2r(const double *in, double *out, long batch, int n, int
     }
 }
 
+/* One-dimensional transforms (Supplement 8.2, the definition itself; Section 5
+ * evaluates batched 1-D transforms of sizes 2..256):
+ *   X_k = sum_{j<len} x_j exp(-2 pi i k j / n),  k in [0, n/2],
+ * the signal zero-padded from len to n samples, only the Hermitian half stored.
+ * in: [batch][len] floats; out: [batch][n/2+1][2] doubles. O(n len) per signal. */
+API void oracle_dft1d_r2c(const float *in, double *out, long batch, int len, int n) {
+    const int nc = n / 2 + 1;
+    const double two_pi = 6.283185307179586476925286766559;
+#pragma omp parallel for schedule(static)
+    for (long p = 0; p < batch; ++p) {
+        const float *xp = in + (size_t)p * len;
+        double *op = out + (size_t)p * nc * 2;
+        for (int k = 0; k < nc; ++k) {
+            double re = 0.0, im = 0.0;
+            for (int j = 0; j < len; ++j) {
+                int m = (int)(((long)k * j) % n);
+                double ang = -two_pi * (double)m / (double)n;
+                re += (double)xp[j] * cos(ang);
+                im += (double)xp[j] * sin(ang);
+            }
+            op[2 * k + 0] = re;
+            op[2 * k + 1] = im;
+        }
+    }
+}
+
+/* Inverse of the above: x_j = scale * Re sum_{k<n} X~_k exp(+2 pi i k j / n) for j < olen,
+ * X~_k = X_k for k <= n/2, conj(X_{n-k}) above (Hermitian extension).
+ * in: [batch][n/2+1][2] doubles; out: [batch][olen] doubles. */
+API void oracle_idft1d_c2r(const double *in, double *out, long batch, int n, int olen,
+                           double scale) {
+    const int nc = n / 2 + 1;
+    const double two_pi = 6.283185307179586476925286766559;
+#pragma omp parallel for schedule(static)
+    for (long p = 0; p < batch; ++p) {
+        const double *sp = in + (size_t)p * nc * 2;
+        double *op = out + (size_t)p * olen;
+        for (int j = 0; j < olen; ++j) {
+            double acc = 0.0;
+            for (int k = 0; k < n; ++k) {
+                double re, im;
+                if (k < nc) { re = sp[2 * k]; im = sp[2 * k + 1]; }
+                else        { re = sp[2 * (n - k)]; im = -sp[2 * (n - k) + 1]; }
+                int m = (int)(((long)k * j) % n);
+                double ang = two_pi * (double)m / (double)n;
+                acc += re * cos(ang) - im * sin(ang);
+            }
+            op[j] = scale * acc;
+        }
+    }
+}
+
 /* Per-bin complex contraction of Table 1's Cgemm row, written as the plain
  * sum: C[b][m][n] = sum_k opA(A[b][m][k]) * opB(B[b][n][k]), conjA / conjB
  * select complex conjugation of that operand (Section 2: the conjugate makes

@@ -6,7 +6,7 @@ The compute path is the CUDA library only -- there is no CPU fallback.
 """
 from . import workloads  # noqa: F401
 from .binding import (  # noqa: F401
-    MATH_AUTO, MATH_FP32, MATH_TF32, FftConvError, Plan, conv_accgrad, conv_bprop, conv_fprop, conv_fprop_noalloc,
+    MATH_AUTO, MATH_FP32, MATH_TF32, TILE_AUTO, FftConvError, Plan, conv_accgrad, conv_bprop, conv_fprop, conv_fprop_noalloc,
     conv_plan, conv_plan_alloc_workspace, conv_plan_destroy, conv_plan_effective_math, conv_plan_pass_math, conv_plan_enable_stage_timing,
     conv_plan_stage_times_ms,
     conv_plan_set_math, conv_plan_set_tiling, conv_plan_tile_basis, conv_plan_set_spectrum_reuse, conv_plan_invalidate_spectra, conv_plan_set_workspace, conv_plan_status, conv_plan_workspace_bytes,

@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libfftconv.so")
 OK = 0
 EINVAL, EUNSUPPORTED, EWORKSPACE, ECUDA, EDEVICE_TIMEOUT = -1, -2, -3, -4, -5
 MATH_AUTO, MATH_FP32, MATH_TF32 = 0, 1, 2
+TILE_AUTO = -1
 
 EXPORTS = (
     "conv_plan", "conv_plan_set_math", "conv_plan_effective_math", "conv_plan_pass_math",

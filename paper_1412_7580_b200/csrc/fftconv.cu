@@ -355,8 +355,53 @@ FFTCONV_API size_t conv_plan_workspace_bytes(const conv_plan_t* plan) {
            (plan->n != plan->n_full ? 0 : fc::big_scratch_bytes(plan->n));
 }
 
+namespace {
+// Plan-time estimate of one training step (three passes) in microseconds, from the bytes each
+// kernel family moves and the rates measured for it on B200 (TB/s = bytes per picosecond):
+// transforms 4.4 (n <= 32), 3.0 (n = 64), 2.2 (n = 128), windowed forward transforms 2.9
+// (1.6 at n = 8, 2.2 at n = 16: the fixed cost per window weighs more),
+// contraction 5.5; plus a fixed cost per launch.  Only used to rank tile bases against each other.
+double estimate_step_us(const conv_plan_s& p) {
+    const bool tiled = p.n != p.n_full;
+    const double fft_rate = p.n <= 32 ? 4.4e6 : (p.n == 64 ? 3.0e6 : 2.2e6);     // bytes per us
+    const double win_rate = p.n >= 32 ? 2.9e6 : (p.n == 16 ? 2.2e6 : 1.6e6);
+    double us = 0.0;
+    for (int pass = 0; pass < 3; ++pass) {
+        const PassDesc d = describe(p, pass);
+        const OperandDesc* ops[3] = {&d.a, &d.b, &d.c};
+        double spectra = 0.0;
+        for (int i = 0; i < 3; ++i) {
+            const OperandDesc& o = *ops[i];
+            const double spec = (double)o.spec.bytes(p.bins);
+            const double real = 4.0 * o.spec.R * o.spec.C * o.h * o.w;
+            const bool windowed_load = tiled && o.win && i < 2;
+            us += (spec + real) / (windowed_load ? win_rate : fft_rate);
+            spectra += spec;
+        }
+        us += spectra / 5.5e6 + 3 * 4.0;
+    }
+    return us;
+}
+}  // namespace
+
 FFTCONV_API int conv_plan_set_tiling(conv_plan_t* plan, int n_tile) {
     if (!plan) return FFTCONV_EINVAL;
+    if (n_tile == FFTCONV_TILE_AUTO) {
+        // keep the basis whose estimated step is shortest (the paper's autotuner measures; this
+        // is a static ranking in the spirit of its one-strategy-per-problem-size cache)
+        if (plan->reuse) return FFTCONV_EUNSUPPORTED;
+        int best = 0;
+        conv_plan_set_tiling(plan, 0);
+        double best_us = estimate_step_us(*plan);
+        const int cand[4] = {8, 16, 32, 64};
+        for (int i = 0; i < 4; ++i) {
+            if (cand[i] >= plan->n_full) break;
+            if (conv_plan_set_tiling(plan, cand[i]) != FFTCONV_OK) continue;
+            const double us = estimate_step_us(*plan);
+            if (us < 0.9 * best_us) { best_us = us; best = cand[i]; }    // tiling must win clearly
+        }
+        return conv_plan_set_tiling(plan, best);
+    }
     if (n_tile == 0 || n_tile == plan->n_full) {
         plan->n = plan->n_full;
     } else {

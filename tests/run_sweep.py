@@ -46,6 +46,8 @@ def main():
     ap.add_argument("--max-gb", type=float, default=40.0, help="skip points needing more device memory")
     ap.add_argument("--out", default=os.path.join(ROOT, "gpurun_out", "sweep.jsonl"))
     ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--tile", default="off", choices=["off", "auto"],
+                    help="auto: let every plan choose a tile basis (spatial tiling, Section 6 of the paper)")
     args = ap.parse_args()
 
     peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -70,6 +72,8 @@ def main():
                 continue
             x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
             p = fc.conv_plan(*s.args())
+            if args.tile == "auto":
+                fc.conv_plan_set_tiling(p, fc.TILE_AUTO)
             ws = fc.conv_plan_alloc_workspace(p)
             eff = fc.conv_plan_effective_math(p)
             xd, wd, dyd = (torch.from_numpy(a).cuda() for a in (x, w, dy))
@@ -103,6 +107,7 @@ def main():
             t_roof_ms = b_fft / bw * 1e3        # byte term of the roofline; flops never bind here
             fr = [t_roof_ms / m for m in ms]
             rec = {"point": s.point, "S": s.S, "f": s.f, "fp": s.fp, "h": s.h, "k": s.kh, "n": s.n,
+                   "tile_basis": fc.conv_plan_tile_basis(p),
                    "math": ["tf32" if t == TOL[2] else "f32" for t in tols], "ok": ok,
                    "max_rel_err": errs, "tol": tols,
                    "ms": ms, "roofline_frac": fr,
