@@ -216,6 +216,23 @@ int fft2d_r2c(const float* in, void* out_c, int batch, int h, int w, int n, void
 int fft2d_c2r(const void* in_c, float* out, int batch, int n, int oh, int ow, float scale,
               int accumulate, void* cuda_stream);
 
+/* Bare batched 1-D real-to-complex transform, n a power of two in [2, 256] (the sizes of the
+ * paper's Section 5.2 / 5.4 evaluation of batched 1-D transforms; definition in Supplement 8.2):
+ *   out[p][k] = sum_{j<len} in[p][j] exp(-2 pi i k j / n),   k in [0, n/2]
+ * in : device [batch][len] fp32, zero-padded implicitly to n samples (len <= n).
+ * out: device [batch][n/2+1] interleaved (re, im) fp32 pairs, 8-byte aligned.
+ * EUNSUPPORTED: n not a power of two in [2, 256]; EINVAL: null pointer, batch < 1, len not in [1, n]. */
+int fft1d_r2c(const float* in, void* out_c, long long batch, int len, int n, void* cuda_stream);
+
+/* Bare batched 1-D complex-to-real inverse transform with crop and scale:
+ *   out[p][j] (+)= scale * Re sum_{k<n} X~[p][k] exp(+2 pi i k j / n),   j < olen,
+ * X~ the Hermitian extension of the stored half (the imaginary parts of bins 0 and n/2 are
+ * ignored); scale = 1/n undoes fft1d_r2c.
+ * in : device [batch][n/2+1] interleaved fp32 pairs, 8-byte aligned.
+ * out: device [batch][olen] fp32; accumulate != 0 adds to it. */
+int fft1d_c2r(const void* in_c, float* out, long long batch, int n, int olen, float scale,
+              int accumulate, void* cuda_stream);
+
 /* Per-bin complex contraction alone (Table 1, the Cgemm row), exposed for
  * testing and profiling: for every bin b,
  *   C[b][m][nn] = sum_k op(A)[b][m][k] * op(B)[b][nn][k]

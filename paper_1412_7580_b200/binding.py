@@ -23,7 +23,7 @@ EXPORTS = (
     "conv_plan_set_workspace", "conv_plan_set_spectrum_reuse", "conv_plan_invalidate_spectra",
     "conv_plan_set_tiling", "conv_plan_tile_basis",
     "conv_fprop", "conv_fprop_noalloc", "conv_bprop", "conv_accgrad", "conv_plan_status",
-    "conv_plan_destroy", "conv_plan_enable_stage_timing", "conv_plan_stage_times_ms", "fft2d_r2c", "fft2d_c2r", "fftconv_bin_contract",
+    "conv_plan_destroy", "conv_plan_enable_stage_timing", "conv_plan_stage_times_ms", "fft2d_r2c", "fft2d_c2r", "fft1d_r2c", "fft1d_c2r", "fftconv_bin_contract",
     "fftconv_status_string", "fftconv_launch_count",
 )
 
@@ -67,6 +67,8 @@ def lib():
         L.conv_plan_stage_times_ms.argtypes = [p, p]
         L.fft2d_r2c.argtypes = [p, p, i, i, i, i, p]
         L.fft2d_c2r.argtypes = [p, p, i, i, i, i, fl, i, p]
+        L.fft1d_r2c.argtypes = [p, p, ctypes.c_longlong, i, i, p]
+        L.fft1d_c2r.argtypes = [p, p, ctypes.c_longlong, i, i, fl, i, p]
         L.fftconv_bin_contract.argtypes = [p, p, p] + [i] * 12 + [p, p]
         L.fftconv_status_string.argtypes = [i]
         L.fftconv_status_string.restype = ctypes.c_char_p
@@ -278,6 +280,21 @@ def fft2d_c2r(in_c, out, n, scale, accumulate=False, stream=None) -> None:
     _check(lib().fft2d_c2r(_dev(in_c, (batch, n, n // 2 + 1, 2), "in_c"), _dev(out, None, "out"),
                            batch, int(n), oh, ow, float(scale), int(bool(accumulate)),
                            _stream_ptr(stream)), "fft2d_c2r")
+
+
+def fft1d_r2c(inp, out_c, n, stream=None) -> None:
+    """inp: [batch, len] float32; out_c: [batch, n/2+1, 2] float32 (re, im)."""
+    batch, ln = inp.shape
+    _check(lib().fft1d_r2c(_dev(inp, None, "in"), _dev(out_c, (batch, n // 2 + 1, 2), "out_c"),
+                           batch, ln, int(n), _stream_ptr(stream)), "fft1d_r2c")
+
+
+def fft1d_c2r(in_c, out, n, scale, accumulate=False, stream=None) -> None:
+    """in_c: [batch, n/2+1, 2] float32; out: [batch, olen] float32."""
+    batch, olen = out.shape
+    _check(lib().fft1d_c2r(_dev(in_c, (batch, n // 2 + 1, 2), "in_c"), _dev(out, None, "out"),
+                           batch, int(n), olen, float(scale), int(bool(accumulate)),
+                           _stream_ptr(stream)), "fft1d_c2r")
 
 
 def fftconv_bin_contract(A, B, C, M, N, K, transA=False, transB=False, conjA=False, conjB=False,

@@ -15,6 +15,7 @@
 #include "cgemm_tc.cuh"
 #include "fft_kernels.cuh"
 #include "fft_big.cuh"
+#include "fft1d.cuh"
 
 #define FFTCONV_API extern "C" __attribute__((visibility("default")))
 
@@ -586,6 +587,34 @@ FFTCONV_API int fft2d_c2r(const void* in_c, float* out, int batch, int n, int oh
     p.scale = scale; p.accumulate = accumulate ? 1 : 0;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return fc::launch_c2r<false>(n, p, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? FFTCONV_OK : FFTCONV_ECUDA;
+}
+
+FFTCONV_API int fft1d_r2c(const float* in, void* out_c, long long batch, int len, int n,
+                          void* cuda_stream) {
+    if (!in || !out_c || batch < 1 || len < 1) return FFTCONV_EINVAL;
+    if (n < 2 || n > 256 || (n & (n - 1)) != 0) return FFTCONV_EUNSUPPORTED;
+    if (len > n) return FFTCONV_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(out_c) & 7) != 0) return FFTCONV_EINVAL;
+    fc::Fft1dParams p{};
+    p.real_in = in; p.spec_out = static_cast<float2*>(out_c);
+    p.batch = batch; p.len = len;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return fc::launch_fft1d(n, p, false, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
+               ? FFTCONV_OK : FFTCONV_ECUDA;
+}
+
+FFTCONV_API int fft1d_c2r(const void* in_c, float* out, long long batch, int n, int olen,
+                          float scale, int accumulate, void* cuda_stream) {
+    if (!in_c || !out || batch < 1 || olen < 1) return FFTCONV_EINVAL;
+    if (n < 2 || n > 256 || (n & (n - 1)) != 0) return FFTCONV_EUNSUPPORTED;
+    if (olen > n) return FFTCONV_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(in_c) & 7) != 0) return FFTCONV_EINVAL;
+    fc::Fft1dParams p{};
+    p.spec_in = static_cast<const float2*>(in_c); p.real_out = out;
+    p.batch = batch; p.len = olen; p.scale = scale; p.accumulate = accumulate ? 1 : 0;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return fc::launch_fft1d(n, p, true, static_cast<cudaStream_t>(cuda_stream)) == cudaSuccess
                ? FFTCONV_OK : FFTCONV_ECUDA;
 }
 
