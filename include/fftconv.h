@@ -59,7 +59,10 @@ typedef enum {
  * once).  Host-only: validates the shape, picks kernels and sizes the
  * workspace.  Needs no GPU.  *out receives the plan; destroy it with
  * conv_plan_destroy.  EINVAL: null out, a count < 1, kh > h, kw > w,
- * n < max(h, w).  EUNSUPPORTED: n not a power of two in [8, 128]. */
+ * n < max(h, w).  EUNSUPPORTED: n not a power of two in [8, 128] -- except that n = 256, 512 or
+ * 1024 is accepted for planes of up to n x n samples as the frame of a spatially tiled plan: the
+ * plan then chooses a tile basis at once (see conv_plan_set_tiling; another basis may be set, tiling
+ * cannot be switched off) and no transform of that size is ever run. */
 int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, int w, int kh, int kw, int n);
 
 /* Select the arithmetic of the per-bin contraction (fftconv_math).  Changes the

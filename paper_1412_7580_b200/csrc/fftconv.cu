@@ -301,6 +301,10 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
 
 }  // namespace
 
+namespace {
+double estimate_step_us(const conv_plan_s& p);
+}
+
 FFTCONV_API int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, int w, int kh,
                           int kw, int n) {
     if (!out) return FFTCONV_EINVAL;
@@ -308,7 +312,9 @@ FFTCONV_API int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, in
     if (S < 1 || f < 1 || fprime < 1 || h < 1 || w < 1 || kh < 1 || kw < 1 || n < 1)
         return FFTCONV_EINVAL;
     if (kh > h || kw > w) return FFTCONV_EINVAL;
-    if (!valid_n(n)) return FFTCONV_EUNSUPPORTED;
+    // bases above 128 exist only as the frame of a tiled plan (planes up to 1024 x 1024)
+    const bool frame_only = (n == 256 || n == 512 || n == 1024);
+    if (!valid_n(n) && !frame_only) return FFTCONV_EUNSUPPORTED;
     if (n < h || n < w) return FFTCONV_EINVAL;
     // plane counts and per-tensor element counts must stay inside 31-bit grids / 63-bit offsets
     const long long planes_max = 1LL << 30;
@@ -325,6 +331,22 @@ FFTCONV_API int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, in
     p->ws = nullptr; p->ws_bytes = 0;
     p->timing = 0; p->timed = false; p->ev_made = false;
     p->reuse = 0; p->cached[0] = p->cached[1] = p->cached[2] = nullptr;
+    if (frame_only) {
+        // pick the tile basis now: the estimate ranks 8..64 against each other (the untiled
+        // candidate does not exist), smallest admissible basis as the fallback
+        int best = 0;
+        double best_us = 0.0;
+        const int cand[4] = {8, 16, 32, 64};
+        for (int i = 0; i < 4; ++i) {
+            if (conv_plan_set_tiling(p, cand[i]) != FFTCONV_OK) continue;
+            const double us = estimate_step_us(*p);
+            if (best == 0 || us < best_us) { best = cand[i]; best_us = us; }
+        }
+        if (best == 0 || conv_plan_set_tiling(p, best) != FFTCONV_OK) {
+            delete p;
+            return FFTCONV_EUNSUPPORTED;
+        }
+    }
     *out = p;
     return FFTCONV_OK;
 }
@@ -392,18 +414,23 @@ FFTCONV_API int conv_plan_set_tiling(conv_plan_t* plan, int n_tile) {
         // is a static ranking in the spirit of its one-strategy-per-problem-size cache)
         if (plan->reuse) return FFTCONV_EUNSUPPORTED;
         int best = 0;
-        conv_plan_set_tiling(plan, 0);
-        double best_us = estimate_step_us(*plan);
+        double best_us = 0.0;
+        if (plan->n_full <= 128) {
+            conv_plan_set_tiling(plan, 0);
+            best_us = estimate_step_us(*plan);
+        }
         const int cand[4] = {8, 16, 32, 64};
         for (int i = 0; i < 4; ++i) {
             if (cand[i] >= plan->n_full) break;
             if (conv_plan_set_tiling(plan, cand[i]) != FFTCONV_OK) continue;
             const double us = estimate_step_us(*plan);
-            if (us < 0.9 * best_us) { best_us = us; best = cand[i]; }    // tiling must win clearly
+            const bool first = (plan->n_full > 128 && best == 0);
+            if (first || us < 0.9 * best_us) { best_us = us; best = cand[i]; }   // tiling must win clearly
         }
         return conv_plan_set_tiling(plan, best);
     }
     if (n_tile == 0 || n_tile == plan->n_full) {
+        if (plan->n_full > 128) return FFTCONV_EUNSUPPORTED;   // such a basis exists only tiled
         plan->n = plan->n_full;
     } else {
         // one-pass transforms only; a tile must produce at least one output sample per axis

@@ -61,7 +61,13 @@ def test_plan_validation(L):
     assert plan(8, 4, 8, 16, 16, 17, 3, 16) == b.EINVAL       # kh > h
     assert plan(8, 4, 8, 16, 16, 3, 3, 8) == b.EINVAL         # n < h
     assert plan(8, 4, 8, 16, 16, 3, 3, 24) == b.EUNSUPPORTED  # not a power of two
-    assert plan(8, 4, 8, 16, 16, 3, 3, 256) == b.EUNSUPPORTED
+    assert plan(8, 4, 8, 16, 16, 3, 3, 2048) == b.EUNSUPPORTED
+    # 256, 512, 1024: accepted as the frame of a tiled plan, which cannot be untiled
+    assert plan(2, 4, 8, 200, 200, 3, 3, 256) == b.OK
+    assert L.conv_plan_tile_basis(h) in (8, 16, 32, 64)
+    assert L.conv_plan_set_tiling(h, 0) == b.EUNSUPPORTED
+    assert L.conv_plan_set_tiling(h, b.TILE_AUTO) == b.OK and L.conv_plan_tile_basis(h) > 0
+    assert L.conv_plan_destroy(h) == b.OK
     assert plan(8, 4, 8, 4, 4, 3, 3, 4) == b.EUNSUPPORTED
     # rectangular planes and kernels are accepted
     assert plan(2, 3, 4, 13, 9, 5, 2, 16) == b.OK

@@ -105,3 +105,36 @@ def test_tiled_matches_untiled_bit_for_bit_when_one_tile_covers_the_plane():
     fc.conv_fprop(p, xd, wd, y)
     torch.cuda.synchronize()
     assert np.array_equal(y.cpu().numpy().astype(np.float64), y16)
+
+
+@pytest.mark.parametrize("dims", [
+    (2, 3, 5, 224, 224, 11, 11, 256),      # an ImageNet-size first layer
+    (1, 6, 4, 200, 180, 3, 5, 256),        # rectangular
+    (1, 2, 3, 300, 290, 7, 7, 512),
+])
+def test_planes_larger_than_the_largest_basis_run_tiled(dims):
+    """n = 256 / 512 / 1024 is only the frame of a tiled plan: the plan picks a tile basis itself."""
+    import torch
+    import oracle
+    import paper_1412_7580_b200 as fc
+    from paper_1412_7580_b200 import workloads as wl
+    s = wl.ConvShape("frame", *dims, cfg=8, point=sum(dims))
+    x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+    p = fc.conv_plan(*s.args())
+    assert fc.conv_plan_tile_basis(p) in (8, 16, 32, 64)
+    fc.conv_plan_set_math(p, fc.MATH_FP32)
+    ws = fc.conv_plan_alloc_workspace(p)
+    ws.view(torch.float32)[64:].fill_(float("nan"))
+    xd, wd, dyd = (torch.from_numpy(a).cuda() for a in (x, w, dy))
+    y = torch.full((s.S, s.fp, s.oh, s.ow), float("nan"), device="cuda")
+    dx = torch.full((s.S, s.f, s.h, s.w), float("nan"), device="cuda")
+    dw = torch.full((s.fp, s.f, s.kh, s.kw), float("nan"), device="cuda")
+    fc.conv_fprop(p, xd, wd, y)
+    fc.conv_bprop(p, dyd, wd, dx)
+    fc.conv_accgrad(p, dyd, xd, dw)
+    torch.cuda.synchronize()
+    assert fc.conv_plan_status(p) == 0
+    assert relerr(y.cpu().numpy().astype(np.float64), oracle.fprop(x, w)) <= 1e-4
+    assert relerr(dx.cpu().numpy().astype(np.float64), oracle.bprop(dy, w, s.h, s.w)) <= 1e-4
+    assert relerr(dw.cpu().numpy().astype(np.float64), oracle.accgrad(dy, x, s.kh, s.kw)) <= 1e-4
+    fc.conv_plan_destroy(p)
