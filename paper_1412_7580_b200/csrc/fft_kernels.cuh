@@ -330,18 +330,26 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             const bool col_ok = (cc < sw) && xx >= 0 && xx < pw.W;
             // 4-byte asynchronous copies; a sample outside the plane is a copy of zero bytes,
             // which writes a zero.  Completion: every thread waits for its own copies, then a
-            // barrier (win_pending, at the top of the tile loop).
+            // barrier (win_pending, at the top of the tile loop).  The row test and the address
+            // are formed once per row sweep; the planes of the tile only advance pointers.
             if (cc < sw) {
-                for (int g = 0; g < gcount; ++g) {
-                    const float* pl0 = base + ((size_t)s * sC + c0 + g) * ((size_t)pw.H * pw.W);
-                    const uint32_t dstp = fk_smem_u32(sIn + g * sh * sw + cc);
-                    for (int r = rr; r < sh; r += G) {
-                        const int yy = y0 + r;
-                        const bool ok = col_ok && yy >= 0 && yy < pw.H;
-                        const float* src = ok ? pl0 + (size_t)yy * pw.W + xx : pl0;
+                const int r_lo = max(0, -y0), r_hi = min(sh, pw.H - y0);    // window rows inside the plane
+                const size_t plane = (size_t)pw.H * pw.W;
+                const float* pl0 = base + ((size_t)s * sC + c0) * plane;
+                const long long off0 = (long long)y0 * pw.W + xx;
+                const uint32_t tile_stride = 4u * (uint32_t)(sh * sw);
+                const uint32_t dst0 = fk_smem_u32(sIn + cc);
+                for (int r = rr; r < sh; r += G) {
+                    const bool ok = col_ok && r >= r_lo && r < r_hi;
+                    const float* src = ok ? pl0 + (off0 + (long long)r * pw.W) : pl0;
+                    const size_t step = ok ? plane : 0;
+                    const int nbytes = ok ? 4 : 0;
+                    uint32_t dstp = dst0 + 4u * (uint32_t)(r * sw);
+                    for (int g = 0; g < gcount; ++g) {
                         asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;"
-                                     ::"r"(dstp + 4u * (uint32_t)(r * sw)), "l"(src), "r"(ok ? 4 : 0)
-                                     : "memory");
+                                     ::"r"(dstp), "l"(src), "r"(nbytes) : "memory");
+                        dstp += tile_stride;
+                        src += step;
                     }
                 }
             }

@@ -381,13 +381,13 @@ FFTCONV_API size_t conv_plan_workspace_bytes(const conv_plan_t* plan) {
 namespace {
 // Plan-time estimate of one training step (three passes) in microseconds, from the bytes each
 // kernel family moves and the rates measured for it on B200 (TB/s = bytes per picosecond):
-// transforms 4.4 (n <= 32), 3.0 (n = 64), 2.2 (n = 128), windowed forward transforms 2.9
-// (1.6 at n = 8, 2.2 at n = 16: the fixed cost per window weighs more),
+// transforms 4.4 (n <= 32), 3.0 (n = 64), 2.2 (n = 128), windowed forward transforms 3.4
+// (2.4 at n = 8: the fixed cost per window weighs more),
 // contraction 5.5; plus a fixed cost per launch.  Only used to rank tile bases against each other.
 double estimate_step_us(const conv_plan_s& p) {
     const bool tiled = p.n != p.n_full;
     const double fft_rate = p.n <= 32 ? 4.4e6 : (p.n == 64 ? 3.0e6 : 2.2e6);     // bytes per us
-    const double win_rate = p.n >= 32 ? 2.9e6 : (p.n == 16 ? 2.2e6 : 1.6e6);
+    const double win_rate = p.n >= 16 ? 3.4e6 : 2.4e6;
     double us = 0.0;
     for (int pass = 0; pass < 3; ++pass) {
         const PassDesc d = describe(p, pass);
