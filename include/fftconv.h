@@ -49,7 +49,7 @@ typedef enum {
 } fftconv_status;
 
 typedef enum {
-    FFTCONV_MATH_AUTO = 0, /* tensor cores unless a bin's result has fewer than 64 elements,
+    FFTCONV_MATH_AUTO = 0, /* tensor cores unless a bin's result has fewer than 128 elements,
                               where the FP32 kernel is as fast and exact                  */
     FFTCONV_MATH_FP32 = 1, /* per-bin contraction with FP32 FFMA                  */
     FFTCONV_MATH_TF32 = 2  /* per-bin contraction on tcgen05 tensor cores, TF32

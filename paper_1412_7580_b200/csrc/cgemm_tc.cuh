@@ -67,7 +67,7 @@ static inline bool tc_shape_supported(int M, int N, int K) {
 // enter the choice.
 static inline bool tc_shape_profitable(int M, int N, int K) {
     (void)K;
-    return (long long)M * N >= 64;
+    return (long long)M * N >= 128;
 }
 
 // ---- PTX wrappers ----------------------------------------------------------

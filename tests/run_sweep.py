@@ -5,7 +5,7 @@ all three passes per point on the GPU, checked against the float64 oracle at a
 seeded sample of output coordinates (the plain definition evaluated element by
 element), with per-pass times and roofline fractions.
 
-    python tests/run_sweep.py --points 1000 --budget-s 1200 --out gpurun_out/sweep.jsonl
+    python tests/run_sweep.py --points 1000 --budget-s 1200 --out sweep.jsonl
 
 Writes one JSON line per finished point and a summary line at the end; points
 are visited in a seeded random order so that a time-boxed run is an unbiased
@@ -44,7 +44,7 @@ def main():
     ap.add_argument("--points", type=int, default=1000)
     ap.add_argument("--budget-s", type=float, default=1200.0)
     ap.add_argument("--max-gb", type=float, default=40.0, help="skip points needing more device memory")
-    ap.add_argument("--out", default=os.path.join(ROOT, "gpurun_out", "sweep.jsonl"))
+    ap.add_argument("--out", default=os.path.join(ROOT, "sweep.jsonl"))
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--tile", default="off", choices=["off", "auto"],
                     help="auto: let every plan choose a tile basis (spatial tiling, Section 6 of the paper)")
@@ -54,7 +54,7 @@ def main():
     bw = (json.load(open(peaks_path))["hbm_gbs"] if os.path.exists(peaks_path) else 6650.0) * 1e9
     pts = wl.sweep_points(args.points)
     order = np.random.default_rng([wl.SEED_ROOT, 55]).permutation(len(pts))
-    os.makedirs(os.path.dirname(args.out), exist_ok=True)
+    os.makedirs(os.path.dirname(os.path.abspath(args.out)), exist_ok=True)
     t_start = time.time()
     done = failed = skipped = 0
     fracs, worst = [], 0.0

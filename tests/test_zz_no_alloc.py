@@ -31,7 +31,7 @@ def _fprop_pair(fc, shape, x, w):
     y_new = torch.full_like(y_ref, float("nan"))
     fc.conv_fprop_noalloc(q, xd, wd, y_new)
     torch.cuda.synchronize()
-    eff = fc.conv_plan_effective_math(q)
+    eff = fc.conv_plan_pass_math(q, 0)       # fprop is pass 0; AUTO math resolves per pass
     fc.conv_plan_destroy(p)
     fc.conv_plan_destroy(q)
     return y_ref.cpu().numpy().astype(np.float64), y_new.cpu().numpy().astype(np.float64), eff
