@@ -80,9 +80,9 @@ int conv_plan_pass_math(const conv_plan_t* plan, int pass);
 
 /* Bytes of device scratch the three passes need: the frequency-domain copies of
  * the two operands and of the result (Section 6 lists the same buffers), in the
- * plan's private frequency-major layout; plans with n = 64 or 128 add the
- * scratch that the transforms of large planes pass their half spectra through
- * between the two 1-D passes (40 and 80 MiB).  0 on a null plan. */
+ * plan's private frequency-major layout; plans with n = 128 add the scratch
+ * that the transforms of large planes pass their half spectra through between
+ * the two 1-D passes (80 MiB).  0 on a null plan. */
 size_t conv_plan_workspace_bytes(const conv_plan_t* plan);
 
 /* Lend the plan `bytes` of device memory at `dev_ptr` (256-byte aligned).  The

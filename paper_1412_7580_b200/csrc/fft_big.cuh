@@ -64,14 +64,23 @@ struct BigGeom {
     static constexpr int NT = BigCfg<N>::NT;                     // teams per CTA
     static constexpr int THREADS = NT * TEAM;
     static constexpr size_t SMEM = NT * INBUF + STAGE_NY;      // one buffer per team + the ky = N/2 staging
+    // The scratch kept in shared memory instead (n = 64: 132 KB, one CTA per SM): rows of N + 2 and
+    // planes of M rows + 2 complex, so that both the rows of one plane and the same row of
+    // adjacent planes start an odd number of 16-byte units apart (conflict-free 16-byte loads).
+    static constexpr int SPITCH = N + 2;
+    static constexpr int SPLANE = M * SPITCH + 2;
+    static constexpr size_t SSCRATCH = (size_t)BIG_G * SPLANE * 8;
+    static constexpr size_t SMEM_SS = SMEM + SSCRATCH;
     static_assert(PLANE <= INBUF && STAGE <= INBUF, "a team's buffer holds a plane, a chunk or a staging tile");
     static_assert((size_t)2 * H * N * 8 <= INBUF, "the exchange buffer fits a team's buffer");
     static_assert(TEAM == 4 * ROWS && KC >= 1 && M % KC == 0, "thread roles");
 };
 
+// n = 64: the scratch fits in shared memory (one CTA per SM); n = 128 needs the global area.
+constexpr bool big_smem_scratch(int n) { return n == 64; }
+
 static inline size_t big_scratch_bytes(int n) {
     if (n == 128) return (size_t)BIG_MAX_SMS * BigCfg<128>::MINB * BigGeom<128>::SCRATCH_PER_CTA;
-    if (n == 64) return (size_t)BIG_MAX_SMS * BigCfg<64>::MINB * BigGeom<64>::SCRATCH_PER_CTA;
     return 0;
 }
 
@@ -214,14 +223,20 @@ __device__ __forceinline__ void big_split4_rows(const float2* rowp, float (&ar)[
 // ---------------------------------------------------------------------------
 // Forward.
 // ---------------------------------------------------------------------------
-template <int N>
-__global__ void __launch_bounds__(BigGeom<N>::THREADS, BigCfg<N>::MINB)
+// SS: the scratch between the two 1-D passes lives in shared memory (fits for n = 64 with one
+// CTA per SM) instead of the CTA-private global area; the row pass then reads it in place.
+template <int N, bool SS>
+__global__ void __launch_bounds__(BigGeom<N>::THREADS, SS ? 1 : BigCfg<N>::MINB)
 r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmNy,
                const FftParams p, float2* __restrict__ scratch_all) {
     using Gm = BigGeom<N>;
     constexpr int M = Gm::M, L = Gm::L, H = Gm::H, G = BIG_G, T = Gm::TEAM, NT = Gm::NT, KC = Gm::KC, PITCH = Gm::PITCH;
+    constexpr int RS = SS ? Gm::SPITCH : N;                // scratch: complex per row
+    constexpr int PS = SS ? Gm::SPLANE : M * N;            // scratch: complex per plane
     extern __shared__ __align__(128) unsigned char fc_smem[];
-    float2* scratch = scratch_all + (size_t)blockIdx.x * (G * M * N);
+    float2* scratch;
+    if constexpr (SS) scratch = reinterpret_cast<float2*>(fc_smem + Gm::SMEM);
+    else scratch = scratch_all + (size_t)blockIdx.x * (G * M * N);
 
     const int team = threadIdx.x / T, tid = threadIdx.x - team * T;      // tid: index inside the team
     unsigned char* buf = fc_smem + (size_t)team * Gm::INBUF;            // the team's buffer
@@ -282,7 +297,10 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
             big_team_sync<T>(team);                           // plane g is in registers: the buffer takes the next one
             if (g + NT < gcount) issue_plane(row, c0, g + NT);
             fk_cp_commit();
-            float2* dst = scratch + (size_t)(g * M) * N + cA;
+            float2* dst = scratch + (size_t)g * PS + cA;
+            auto put = [&](float2* a, float2 v) {
+                if constexpr (SS) *a = v; else big_st2(a, v, keep);
+            };
             if (live) {
                 if (q2 == 0) {
                     // bins k = 2i; rows ky = 0 and ky = N/2 are real and share row 0 as (re, im)
@@ -290,19 +308,19 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                     rfft_half_finish<N, 0>(ar, ai, [&](auto I, float re, float im) {
                         constexpr int i = decltype(I)::value;
                         if constexpr (i == 0) x0 = re;
-                        else if constexpr (i == H) big_st2(dst, make_float2(x0, re), keep);
-                        else big_st2(dst + (size_t)(2 * i) * N, make_float2(re, im), keep);
+                        else if constexpr (i == H) put(dst, make_float2(x0, re));
+                        else put(dst + (size_t)(2 * i) * RS, make_float2(re, im));
                     });
                 } else {
                     rfft_half_finish<N, 1>(ar, ai, [&](auto I, float re, float im) {
                         constexpr int i = decltype(I)::value;
-                        big_st2(dst + (size_t)(2 * i + 1) * N, make_float2(re, im), keep);
+                        put(dst + (size_t)(2 * i + 1) * RS, make_float2(re, im));
                     });
                 }
             } else {
                 static_for<H>([&](auto I) {
                     constexpr int i = decltype(I)::value;
-                    big_st2(dst + (size_t)(2 * i + q2) * N, make_float2(0.0f, 0.0f), keep);
+                    put(dst + (size_t)(2 * i + q2) * RS, make_float2(0.0f, 0.0f));
                 });
             }
         }
@@ -312,12 +330,18 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
         // ---- B: row transforms; chunks team, team + NT, .. --------------------------------
         constexpr int CHUNKS = M / KC;
         for (int ci = team; ci < CHUNKS; ci += NT) {
-            issue_chunk(ci);
-            fk_cp_commit();
-            fk_cp_wait<0>();
-            big_team_sync<T>(team);                           // chunk ci has landed for the team
             float ar[L], ai[L];
-            const float2* rowp = reinterpret_cast<const float2*>(buf) + rB * PITCH;
+            const float2* rowp;
+            if constexpr (SS) {
+                // read the row in place: row rB of the chunk is (plane rB % 8, ky = ci KC + rB / 8)
+                rowp = scratch + (size_t)(rB & (G - 1)) * PS + (size_t)(ci * KC + (rB >> 3)) * RS;
+            } else {
+                issue_chunk(ci);
+                fk_cp_commit();
+                fk_cp_wait<0>();
+                big_team_sync<T>(team);                       // chunk ci has landed for the team
+                rowp = reinterpret_cast<const float2*>(buf) + rB * PITCH;
+            }
             if (q4 == 0)      big_split4_rows<N, false, 0>(rowp, ar, ai);
             else if (q4 == 1) big_split4_rows<N, false, 1>(rowp, ar, ai);
             else if (q4 == 2) big_split4_rows<N, false, 2>(rowp, ar, ai);
@@ -368,15 +392,19 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
 // ---------------------------------------------------------------------------
 // Inverse.
 // ---------------------------------------------------------------------------
-template <int N>
-__global__ void __launch_bounds__(BigGeom<N>::THREADS, BigCfg<N>::MINB)
+template <int N, bool SS>
+__global__ void __launch_bounds__(BigGeom<N>::THREADS, SS ? 1 : BigCfg<N>::MINB)
 c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmNy,
                const FftParams p, float2* __restrict__ scratch_all) {
     using Gm = BigGeom<N>;
     constexpr int M = Gm::M, L = Gm::L, H = Gm::H, G = BIG_G, T = Gm::TEAM, NT = Gm::NT, KC = Gm::KC, PITCH = Gm::PITCH;
+    constexpr int RS = SS ? Gm::SPITCH : N;
+    constexpr int PS = SS ? Gm::SPLANE : M * N;
     extern __shared__ __align__(128) unsigned char fc_smem[];
     __shared__ __align__(8) unsigned long long bar_storage[NT];
-    float2* scratch = scratch_all + (size_t)blockIdx.x * (G * M * N);
+    float2* scratch;
+    if constexpr (SS) scratch = reinterpret_cast<float2*>(fc_smem + Gm::SMEM);
+    else scratch = scratch_all + (size_t)blockIdx.x * (G * M * N);
 
     const int team = threadIdx.x / T, tid = threadIdx.x - team * T;
     unsigned char* buf = fc_smem + (size_t)team * Gm::INBUF;
@@ -439,6 +467,14 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
             }
             big_team_sync<T>(team);                           // staging tile in registers: the buffer takes the rows
             cfft<L, true>(ar, ai);                         // ar/ai[m] = value at column 4m + q4
+            if constexpr (SS) {
+                // straight into the shared-memory scratch: row rB is (plane rB % 8, ky = ci KC + rB / 8)
+                float2* dst = scratch + (size_t)(rB & (G - 1)) * PS + (size_t)(ci * KC + (rB >> 3)) * RS + q4;
+                static_for<L>([&](auto Mm) {
+                    constexpr int m = decltype(Mm)::value;
+                    dst[4 * m] = make_float2(ar[m], ai[m]);
+                });
+            } else {
             float2* sRows = reinterpret_cast<float2*>(buf);
             float2* dst = sRows + rB * PITCH + q4;
             static_for<L>([&](auto Mm) {
@@ -455,6 +491,7 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 big_st4(reinterpret_cast<float4*>(scratch + ((size_t)(g * M + ky) * N + 2 * pc)), v, keep);
             }
             big_team_sync<T>(team);                           // the buffer is free for the next chunk
+            }
         }
         __syncthreads();                                   // the scratch is complete for this CTA
 
@@ -462,10 +499,11 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
         float2* sX = reinterpret_cast<float2*>(buf);
         for (int g = team; g < gcount; g += NT) {
             float er[H], ei[H];
-            const float2* src = scratch + (size_t)(g * M) * N + cA;
+            const float2* src = scratch + (size_t)g * PS + cA;
             auto X = [&](auto K) -> float2 {
                 constexpr int k = decltype(K)::value;
-                return big_ld2(src + (size_t)k * N, keep);
+                if constexpr (SS) return src[(size_t)k * RS];
+                else return big_ld2(src + (size_t)k * N, keep);
             };
             if (q2 == 0) irfft_half<N, 0>(X, er, ei);
             else         irfft_half<N, 1>(X, er, ei);
@@ -518,8 +556,16 @@ static cudaError_t launch_r2c_big(FftParams p, float* scratch, size_t scratch_by
     memset(&tmny, 0, sizeof(tmny));
     if (!big_make_map<N>(&tm, p.spec_out, p, Gm::KC) || !big_make_map<N>(&tmny, p.spec_out, p, 1))
         return cudaErrorInvalidValue;
-    auto kern = r2c_big_kernel<N>;
     int grid = 0;
+    if constexpr (big_smem_scratch(N)) {
+        (void)scratch; (void)scratch_bytes;
+        auto kern = r2c_big_kernel<N, true>;
+        cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), Gm::THREADS, Gm::SMEM_SS, p.num_tiles, &grid);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, Gm::THREADS, Gm::SMEM_SS, st>>>(tm, tmny, p, nullptr);
+        return cudaGetLastError();
+    } else {
+    auto kern = r2c_big_kernel<N, false>;
     cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), Gm::THREADS, Gm::SMEM, p.num_tiles, &grid);
     if (e != cudaSuccess) return e;
     const long long fit = (long long)(scratch_bytes / Gm::SCRATCH_PER_CTA);
@@ -527,6 +573,7 @@ static cudaError_t launch_r2c_big(FftParams p, float* scratch, size_t scratch_by
     if (grid > fit) grid = (int)fit;
     kern<<<grid, Gm::THREADS, Gm::SMEM, st>>>(tm, tmny, p, reinterpret_cast<float2*>(scratch));
     return cudaGetLastError();
+    }
 }
 
 template <int N>
@@ -538,9 +585,17 @@ static cudaError_t launch_c2r_big(FftParams p, float* scratch, size_t scratch_by
     memset(&tmny, 0, sizeof(tmny));
     if (!big_make_map<N>(&tm, p.spec_in, p, Gm::KC) || !big_make_map<N>(&tmny, p.spec_in, p, 1))
         return cudaErrorInvalidValue;
-    auto kern = c2r_big_kernel<N>;
-    constexpr size_t SMEM = Gm::SMEM;
     int grid = 0;
+    if constexpr (big_smem_scratch(N)) {
+        (void)scratch; (void)scratch_bytes;
+        auto kern = c2r_big_kernel<N, true>;
+        cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), Gm::THREADS, Gm::SMEM_SS, p.num_tiles, &grid);
+        if (e != cudaSuccess) return e;
+        kern<<<grid, Gm::THREADS, Gm::SMEM_SS, st>>>(tm, tmny, p, nullptr);
+        return cudaGetLastError();
+    } else {
+    auto kern = c2r_big_kernel<N, false>;
+    constexpr size_t SMEM = Gm::SMEM;
     cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), Gm::THREADS, SMEM, p.num_tiles, &grid);
     if (e != cudaSuccess) return e;
     const long long fit = (long long)(scratch_bytes / Gm::SCRATCH_PER_CTA);
@@ -548,6 +603,7 @@ static cudaError_t launch_c2r_big(FftParams p, float* scratch, size_t scratch_by
     if (grid > fit) grid = (int)fit;
     kern<<<grid, Gm::THREADS, SMEM, st>>>(tm, tmny, p, reinterpret_cast<float2*>(scratch));
     return cudaGetLastError();
+    }
 }
 
 // Which plane sizes take the two-pass kernels.  n = 64 can run on either family; the
