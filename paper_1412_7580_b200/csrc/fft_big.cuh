@@ -220,6 +220,12 @@ __device__ __forceinline__ void big_split4_rows(const float2* rowp, float (&ar)[
     });
 }
 
+#ifdef FC_EXP_TIMELINE
+#define BIG_TICK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { long long t_ = clock64(); fc_timeline[i] += t_ - tl_last; tl_last = t_; } } while (0)
+#else
+#define BIG_TICK(i) do { } while (0)
+#endif
+
 // ---------------------------------------------------------------------------
 // Forward.
 // ---------------------------------------------------------------------------
@@ -272,17 +278,31 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
     };
 
     bool store_pending = false;
+    bool team_store_pending = false;        // SS: the team's last store may still be reading its buffer
+#ifdef FC_EXP_TIMELINE
+    long long tl_last = clock64();
+#endif
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
         const int row = tile / tpr, tcol = tile - row * tpr;
         const int c0 = tcol * G;
         const int gcount = min(G, p.C - c0);
 
         // ---- A: column transforms; planes team, team + NT, .. ----------------------------
+        if constexpr (SS) {
+            if (team_store_pending) {
+                if (tid == 0) fk_bulk_wait_read();
+                big_team_sync<T>(team);                       // the buffer takes a plane again
+                team_store_pending = false;
+            }
+        }
+        BIG_TICK(0);
         if (team < gcount) issue_plane(row, c0, team);
         fk_cp_commit();
         for (int g = team; g < gcount; g += NT) {
+            BIG_TICK(1);
             fk_cp_wait<0>();
             big_team_sync<T>(team);                           // plane g has landed for the team
+            BIG_TICK(2);
             const float* pl = reinterpret_cast<const float*>(buf) + cA;
             float ar[H], ai[H];
             const bool live = cA < w;
@@ -294,9 +314,11 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 if (q2 == 0) rfft_half_split<N, 0>(x, ar, ai);
                 else         rfft_half_split<N, 1>(x, ar, ai);
             }
+            BIG_TICK(3);
             big_team_sync<T>(team);                           // plane g is in registers: the buffer takes the next one
             if (g + NT < gcount) issue_plane(row, c0, g + NT);
             fk_cp_commit();
+            BIG_TICK(4);
             float2* dst = scratch + (size_t)g * PS + cA;
             auto put = [&](float2* a, float2 v) {
                 if constexpr (SS) *a = v; else big_st2(a, v, keep);
@@ -324,8 +346,10 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 });
             }
         }
+        BIG_TICK(5);
         fk_cp_wait<0>();
         __syncthreads();                                   // the scratch is complete
+        BIG_TICK(6);
 
         // ---- B: row transforms; chunks team, team + NT, .. --------------------------------
         constexpr int CHUNKS = M / KC;
@@ -346,7 +370,14 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
             else if (q4 == 1) big_split4_rows<N, false, 1>(rowp, ar, ai);
             else if (q4 == 2) big_split4_rows<N, false, 2>(rowp, ar, ai);
             else              big_split4_rows<N, false, 3>(rowp, ar, ai);
+            BIG_TICK(7);
+            if constexpr (SS) {
+                // the rows were read in place; the team's buffer is still the previous staging
+                // tile until its store has been read out
+                if (tid == 0 && team_store_pending) fk_bulk_wait_read();
+            }
             big_team_sync<T>(team);                           // the chunk is in registers: the buffer becomes the staging tile
+            BIG_TICK(8);
             cfft<L, false>(ar, ai);                        // ar/ai[m] = F[kx = 4m + q4]
             float* sStage = reinterpret_cast<float*>(buf);
             float* o = sStage + q4 * Gm::ROWS + rB;
@@ -373,18 +404,23 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                     b[kp * G] = xnr; b[(N + kp) * G] = -xni;
                 }
             }
+            BIG_TICK(9);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             big_team_sync<T>(team);
+            BIG_TICK(10);
             if (tid == 0) {
                 fk_tma_store_4d(&tmS, fk_smem_u32(sStage), c0, row, ci * KC, 0, stream);
                 if (ci == 0) fk_tma_store_4d(&tmNy, fk_smem_u32(sNy), c0, row, M, 0, stream);
                 fk_bulk_commit();
-                fk_bulk_wait_read();                       // the buffer may be overwritten after this
+                if constexpr (!SS) fk_bulk_wait_read();    // the buffer may be overwritten after this
             }
             store_pending = true;
-            big_team_sync<T>(team);
+            team_store_pending = true;
+            if constexpr (!SS) big_team_sync<T>(team);
+            BIG_TICK(11);
         }
         __syncthreads();                                   // both teams are done with the scratch
+        BIG_TICK(12);
     }
     if (tid == 0 && store_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }

@@ -215,7 +215,8 @@ __device__ __forceinline__ void load_split_narrow(Load&& load, int live, float (
 }
 
 // Measurement builds (never the shipped library; results are wrong or partial):
-//   -DFC_EXP_TIMELINE  cycle counts per phase of the forward tile loop (CTA 0, thread 0);
+//   -DFC_EXP_TIMELINE  cycle counts per phase of the forward tile loops (CTA 0, thread 0), read
+//                      back through fftconv_debug_timeline (exported by such builds only);
 //   -DFC_EXP_NOMATH    (fft_core.cuh) the butterflies are skipped: data movement only;
 //   -DFC_EXP_TMAONLY   the TMA-staged kernels only move their tiles (input copy, spectrum
 //                      tile load / store), no shared-memory passes and no arithmetic.

@@ -698,3 +698,17 @@ FFTCONV_API const char* fftconv_status_string(int status) {
 FFTCONV_API unsigned long long fftconv_launch_count(void) {
     return g_launches.load(std::memory_order_relaxed);
 }
+
+#ifdef FC_EXP_TIMELINE
+// Measurement builds only: cycle counts per phase of a forward tile loop (CTA 0, thread 0),
+// accumulated since the last reset.
+FFTCONV_API int fftconv_debug_timeline(long long* out16, int reset) {
+    if (out16 && cudaMemcpyFromSymbol(out16, fc::fc_timeline, sizeof(long long) * 16) != cudaSuccess)
+        return FFTCONV_ECUDA;
+    if (reset) {
+        long long zero[16] = {0};
+        if (cudaMemcpyToSymbol(fc::fc_timeline, zero, sizeof(zero)) != cudaSuccess) return FFTCONV_ECUDA;
+    }
+    return FFTCONV_OK;
+}
+#endif
