@@ -138,3 +138,28 @@ def test_planes_larger_than_the_largest_basis_run_tiled(dims):
     assert relerr(dx.cpu().numpy().astype(np.float64), oracle.bprop(dy, w, s.h, s.w)) <= 1e-4
     assert relerr(dw.cpu().numpy().astype(np.float64), oracle.accgrad(dy, x, s.kh, s.kw)) <= 1e-4
     fc.conv_plan_destroy(p)
+
+
+@pytest.mark.parametrize("dims,n_tile", [((16, 64, 64, 128, 128, 3, 3, 128), 32),
+                                         ((32, 96, 64, 64, 64, 5, 5, 64), 16)])
+def test_tiled_layers_at_benchmark_scale_sampled(dims, n_tile):
+    """Hundreds of thousands of windows in the launch configuration `bench.py --tile` times:
+    sampled output coordinates against the plain definition, plus the adjoint identity on the
+    full GPU tensors."""
+    import oracle
+    from paper_1412_7580_b200 import workloads as wl
+    s = wl.ConvShape("tiled_big", *dims, cfg=8, point=sum(dims))
+    x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+    y, dx, dw, eff = run_tiled(s, n_tile, x, w, dy, 0)
+    for got in (y, dx, dw):
+        assert np.all(np.isfinite(got))
+    cy = wl.sample_coords(y.shape, 3000, seed=11)
+    assert relerr(y[cy[:, 0], cy[:, 1], cy[:, 2], cy[:, 3]], oracle.fprop_at(x, w, cy)) <= TOL[eff[0]]
+    cx = wl.sample_coords(dx.shape, 3000, seed=12)
+    assert relerr(dx[cx[:, 0], cx[:, 1], cx[:, 2], cx[:, 3]], oracle.bprop_at(dy, w, s.h, s.w, cx)) <= TOL[eff[1]]
+    cw = wl.sample_coords(dw.shape, 200, seed=13)
+    assert relerr(dw[cw[:, 0], cw[:, 1], cw[:, 2], cw[:, 3]], oracle.accgrad_at(dy, x, s.kh, s.kw, cw)) <= TOL[eff[2]]
+    tol = max(TOL[e] for e in eff)
+    a = float(np.sum(y * dy)); b = float(np.sum(dx * x)); c = float(np.sum(dw * w))
+    scale = np.sqrt(float(np.sum(y * y)) * float(np.sum(dy.astype(np.float64) ** 2)))
+    assert abs(a - b) <= 10 * tol * scale and abs(a - c) <= 10 * tol * scale
