@@ -676,18 +676,25 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
 // ---------------------------------------------------------------------------
 // Inverse: half spectra -> cropped, scaled real planes.
 // ---------------------------------------------------------------------------
-template <int N, int G, int LAYOUT, int MINB, bool WIN = false>
+// DB: two staging tiles, so that the load of the tile after the next one is issued as soon as
+// a tile has been pulled into registers and the TMA never waits for the CTA (used where only
+// one CTA is resident per SM and a tile's load takes longer than its arithmetic).
+template <int N, int G, int LAYOUT, int MINB, bool WIN = false, bool DB = false>
 __global__ void __launch_bounds__(N* G, MINB)
 c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
     constexpr int T = N * G, NC = N / 2 + 1, M = N / 2, HALF = T / 2, B = N * NC;
     constexpr int PW = MidGeom<N, G>::PW, P = MidGeom<N, G>::P;
     constexpr bool TMA = (LAYOUT == LAYOUT_FREQ_TMA);
     constexpr int D = tma_bins_per_box(N);
+    static_assert(!DB || TMA, "double-buffered staging needs the TMA layout");
+    constexpr int STAGE_FLOATS = 2 * B * G;
     extern __shared__ __align__(128) unsigned char fc_smem[];
     float2* sMid = reinterpret_cast<float2*>(fc_smem);
-    float* sStage = reinterpret_cast<float*>(fc_smem + MidGeom<N, G>::BYTES);
-    __shared__ __align__(8) unsigned long long bar_storage;
-    const uint32_t bar = fk_smem_u32(&bar_storage);
+    float* sStage0 = reinterpret_cast<float*>(fc_smem + MidGeom<N, G>::BYTES);
+    float* sStage = sStage0;
+    __shared__ __align__(8) unsigned long long bar_storage[2];
+    const uint32_t bar0 = fk_smem_u32(&bar_storage[0]);
+    uint32_t bar = bar0;
 
     const int tid = threadIdx.x;
     const int hc = p.h, wc = p.w, hw = hc * wc;
@@ -706,24 +713,34 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
     constexpr int NB = 2 * B / D;
     static_assert(!TMA || NB <= 32, "one lane per TMA box");
     const bool is_fetcher = (tid >= T - 32);
-    auto fetch_tile = [&](int row, int tcol) {      // called by the whole last warp
-        if ((tid & 31) == 0) fk_mbar_expect_tx(bar, (uint32_t)(2 * B * G * 4));
+    auto fetch_into = [&](int row, int tcol, float* stage, uint32_t barrier) {   // whole last warp
+        if ((tid & 31) == 0) fk_mbar_expect_tx(barrier, (uint32_t)(2 * B * G * 4));
         __syncwarp();
         if ((tid & 31) < NB) {
             const int b0 = (tid & 31) * D;
-            fk_tma_load_3d(fk_smem_u32(sStage + (size_t)b0 * G), &tmS, tcol * G, row, b0, bar);
+            fk_tma_load_3d(fk_smem_u32(stage + (size_t)b0 * G), &tmS, tcol * G, row, b0, barrier);
         }
     };
-    uint32_t phase = 0;
+    auto fetch_tile = [&](int row, int tcol) { fetch_into(row, tcol, sStage, bar); };
+    uint32_t phase = 0;             // DB: bit b is the phase of buffer b's barrier
     int row = blockIdx.x / tpr, tcol = blockIdx.x - (blockIdx.x / tpr) * tpr;
     if constexpr (TMA) {
         if (tid == 0) {
-            fk_mbar_init(bar, 1);
+            fk_mbar_init(bar0, 1);
+            if (DB) fk_mbar_init(bar0 + 8u, 1);
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         __syncthreads();
         if (is_fetcher && blockIdx.x < p.num_tiles) fetch_tile(row, tcol);
+        if constexpr (DB) {
+            if (is_fetcher && blockIdx.x + gridDim.x < p.num_tiles) {
+                int r1 = row, c1 = tcol;
+                advance(r1, c1);
+                fetch_into(r1, c1, sStage0 + STAGE_FLOATS, bar0 + 8u);
+            }
+        }
     }
+    int buf = 0;
 
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, advance(row, tcol)) {
         const int c0 = tcol * G;
@@ -734,8 +751,15 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
         // 1. row transforms (along kx): thread = (half q, row kyp, plane gB)
         float ar[M], ai[M];
         if constexpr (TMA) {
+            if constexpr (DB) {
+                sStage = sStage0 + buf * STAGE_FLOATS;
+                bar = bar0 + 8u * (uint32_t)buf;
+                if (!fk_mbar_wait(bar, (phase >> buf) & 1u)) return;
+                phase ^= (1u << buf);
+            } else {
             if (!fk_mbar_wait(bar, phase)) return;
             phase ^= 1u;
+            }
 #ifdef FC_EXP_TMAONLY
             __syncthreads();
             if (is_fetcher && tile + (int)gridDim.x < p.num_tiles) fetch_tile(row_n, tcol_n);
@@ -770,7 +794,17 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             if (q == 0) load_split<N, true, 0>(load, ar, ai);
             else        load_split<N, true, 1>(load, ar, ai);
             __syncthreads();        // staging tile consumed; previous tile's step 2 is done with sMid
+            if constexpr (DB) {
+                // this buffer takes the tile after the next one
+                if (is_fetcher && tile + 2 * (int)gridDim.x < p.num_tiles) {
+                    int r2 = row_n, c2 = tcol_n;
+                    advance(r2, c2);
+                    fetch_tile(r2, c2);
+                }
+                buf ^= 1;
+            } else {
             if (is_fetcher && tile + (int)gridDim.x < p.num_tiles) fetch_tile(row_n, tcol_n);
+            }
         } else {
             if (gB < gcount) {
                 const size_t mat = (size_t)p.R * p.ld;
@@ -1018,23 +1052,27 @@ static cudaError_t launch_r2c_n(FftParams pa, const FftParams* pb_in, cudaStream
     return cudaGetLastError();
 }
 
+// Plane sizes whose inverse transform double-buffers its staging tile (one resident CTA per SM).
+template <int N> struct C2rDoubleBuffer { static constexpr bool value = (N == 64); };
+
 template <int N, bool FREQ>
 static cudaError_t launch_c2r_n(FftParams p, cudaStream_t st) {
     using Cfg = FftCfg<N>;
     constexpr int G = Cfg::G;
     constexpr int LAYOUT = !FREQ ? LAYOUT_BARE : (Cfg::TMA ? LAYOUT_FREQ_TMA : LAYOUT_FREQ_DIRECT);
+    constexpr bool DB = C2rDoubleBuffer<N>::value && LAYOUT == LAYOUT_FREQ_TMA;
     if (!fill_tiling<G>(p)) return cudaErrorInvalidValue;
     p.in_bytes = 0;
     size_t smem = MidGeom<N, G>::BYTES;
     CUtensorMap tm;
     memset(&tm, 0, sizeof(tm));
     if (LAYOUT == LAYOUT_FREQ_TMA) {
-        smem += (size_t)2 * N * (N / 2 + 1) * G * sizeof(float);
+        smem += (size_t)(DB ? 2 : 1) * 2 * N * (N / 2 + 1) * G * sizeof(float);
         if (!make_spec_map<N, G>(&tm, p.spec_in, p)) return cudaErrorInvalidValue;
     }
     if (p.win && LAYOUT != LAYOUT_FREQ_TMA) return cudaErrorInvalidValue;
-    auto kern = (p.win && LAYOUT == LAYOUT_FREQ_TMA) ? c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV, LAYOUT == LAYOUT_FREQ_TMA>
-                                                     : c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV, false>;
+    auto kern = (p.win && LAYOUT == LAYOUT_FREQ_TMA) ? c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV, LAYOUT == LAYOUT_FREQ_TMA, DB>
+                                                     : c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV, false, DB>;
     int grid = 0;
     cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), N * G, smem, p.num_tiles, &grid);
     if (e != cudaSuccess) return e;
