@@ -1052,8 +1052,10 @@ static cudaError_t launch_r2c_n(FftParams pa, const FftParams* pb_in, cudaStream
     return cudaGetLastError();
 }
 
-// Plane sizes whose inverse transform double-buffers its staging tile (one resident CTA per SM).
-template <int N> struct C2rDoubleBuffer { static constexpr bool value = (N == 64); };
+// Plane sizes whose inverse transform double-buffers its staging tile.
+// Measured on B200: n = 64 (one resident CTA) 76-79 -> 72 us on the large-kernel layer, n = 16 44 -> 41 us
+// on the deep layer's accGrad; n = 32 loses a resident CTA to the second tile and gains nothing.
+template <int N> struct C2rDoubleBuffer { static constexpr bool value = (N == 64 || N == 16); };
 
 template <int N, bool FREQ>
 static cudaError_t launch_c2r_n(FftParams p, cudaStream_t st) {
