@@ -18,6 +18,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <stdint.h>
 
 #include "fft_core.cuh"
 
@@ -45,6 +46,14 @@ template <int N> struct F1Cfg {
     static constexpr int SMEM = TB * (PITCH_C * 8 > PITCH_R * 4 ? PITCH_C * 8 : PITCH_R * 4);
 };
 
+// Asynchronous copy of BYTES (4 or 8) from global to shared memory.
+template <int BYTES>
+__device__ __forceinline__ void f1_cp_async(void* smem_dst, const void* gmem_src) {
+    asm volatile("cp.async.ca.shared.global [%0], [%1], %2;"
+                 ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst))), "l"(gmem_src), "n"(BYTES)
+                 : "memory");
+}
+
 // cos and sin of 2 pi k / n for a run-time k (post- and pre-pass of the split transforms)
 __device__ __forceinline__ void f1_twiddle(int k, int n, float& c, float& s) {
     sincospif(2.0f * (float)k / (float)n, &s, &c);
@@ -69,11 +78,12 @@ fft1d_r2c_kernel(const Fft1dParams p) {
         int r = tid / len, j = tid - r * len;
         const int dr = F1_THREADS / len, dj = F1_THREADS - dr * len;
         for (int idx = tid; idx < cnt * len; idx += F1_THREADS) {
-            sR[r * pr + j] = __ldg(src + idx);
+            f1_cp_async<4>(sR + r * pr + j, src + idx);     // asynchronous: the loop only issues
             r += dr; j += dj;
             if (j >= len) { j -= len; ++r; }
         }
     }
+    asm volatile("cp.async.wait_all;" ::: "memory");
     __syncthreads();
 
     if constexpr (C::TPT == 1) {
@@ -173,9 +183,10 @@ fft1d_c2r_kernel(const Fft1dParams p) {
         const float2* src = p.spec_in + t0 * NC;
         for (int idx = tid; idx < cnt * NC; idx += F1_THREADS) {
             const int r = idx / NC, k = idx - r * NC;
-            sC[r * PC + k] = __ldg(src + idx);
+            f1_cp_async<8>(sC + r * PC + k, src + idx);
         }
     }
+    asm volatile("cp.async.wait_all;" ::: "memory");
     __syncthreads();
 
     if constexpr (C::TPT == 1) {
