@@ -14,6 +14,8 @@
 
 #include <cuda_runtime.h>
 
+#include "dep_launch.cuh"
+
 namespace fc {
 
 struct GemmParams {
@@ -24,6 +26,7 @@ struct GemmParams {
     int lda, ldb, ldc;
     int transA, transB;   // operand stored [K][rows] instead of [rows][K]
     int conjA, conjB;     // use the complex conjugate of the operand
+    int overlap;          // host only: launch as a programmatic dependent of the previous kernel
 };
 
 constexpr int FG_BM = 64, FG_BN = 64, FG_BK = 16, FG_PAD = 4, FG_T = 256;
@@ -32,6 +35,8 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
     __shared__ __align__(16) float sA[2][FG_BK][FG_BM + FG_PAD];
     __shared__ __align__(16) float sB[2][FG_BK][FG_BN + FG_PAD];
 
+    dep_trigger();
+    dep_wait();                     // no global access above this line
     const int tid = threadIdx.x;
     const int bin = blockIdx.z;
     const int m_blk = blockIdx.y * FG_BM, n_blk = blockIdx.x * FG_BN;
@@ -151,8 +156,7 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
 static cudaError_t launch_cgemm_ffma(const GemmParams& p, cudaStream_t st) {
     dim3 grid((p.N + FG_BN - 1) / FG_BN, (p.M + FG_BM - 1) / FG_BM, p.bins);
     if (grid.y > 65535u || grid.z > 65535u) return cudaErrorInvalidValue;
-    cgemm_ffma_kernel<<<grid, FG_T, 0, st>>>(p);
-    return cudaGetLastError();
+    return dep_launch(p.overlap != 0, cgemm_ffma_kernel, grid, dim3(FG_T), 0, st, p);
 }
 
 }  // namespace fc

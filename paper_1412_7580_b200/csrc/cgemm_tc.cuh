@@ -36,6 +36,7 @@
 
 #include "cgemm_ffma.cuh"
 #include "tma_util.cuh"
+#include "dep_launch.cuh"
 
 namespace fc {
 
@@ -201,6 +202,7 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
+    dep_trigger();
     if (tid == 0) {
         for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), 128); }
@@ -217,6 +219,7 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    dep_wait();                     // no global access above this line
 
     const int num_tiles = p.bins * p.m_tiles * p.n_tiles;
     auto give_up = [&]() {
@@ -424,8 +427,7 @@ static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStrea
     const long long tiles = (long long)p.bins * p.m_tiles * p.n_tiles;
     if (tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    kern<<<grid, TC_THREADS, TC_SMEM_BYTES, st>>>(tmA, tmB, tmC, p);
-    return cudaGetLastError();
+    return dep_launch(g.overlap != 0, kern, dim3(grid), dim3(TC_THREADS), TC_SMEM_BYTES, st, tmA, tmB, tmC, p);
 }
 
 static cudaError_t launch_cgemm_tc(const GemmParams& g, int* status, cudaStream_t st) {

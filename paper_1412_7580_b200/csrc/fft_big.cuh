@@ -252,6 +252,8 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
     const int h = p.h, w = p.w, hw = h * w;
     const int tpr = p.tiles_per_row;
     const uint64_t keep = big_policy_keep(), stream = big_policy_stream();
+    dep_trigger();
+    dep_wait();                     // no global access above this line
 
     // copy of one real plane into the team's buffer
     auto issue_plane = [&](int row, int c0, int g) {
@@ -455,11 +457,13 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
     constexpr int CHUNKS = M / KC;
     const uint64_t keep = big_policy_keep(), stream = big_policy_stream();
 
+    dep_trigger();
     if (tid == 0) {
         fk_mbar_init(bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    dep_wait();                     // no global access above this line
     uint32_t phase = 0u;
     bool dead = false;          // a load never landed: keep walking through the barriers, stop waiting
 
@@ -598,8 +602,7 @@ static cudaError_t launch_r2c_big(FftParams p, float* scratch, size_t scratch_by
         auto kern = r2c_big_kernel<N, true>;
         cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), Gm::THREADS, Gm::SMEM_SS, p.num_tiles, &grid);
         if (e != cudaSuccess) return e;
-        kern<<<grid, Gm::THREADS, Gm::SMEM_SS, st>>>(tm, tmny, p, nullptr);
-        return cudaGetLastError();
+        return dep_launch(false, kern, dim3(grid), dim3(Gm::THREADS), Gm::SMEM_SS, st, tm, tmny, p, (float2*)nullptr);
     } else {
     auto kern = r2c_big_kernel<N, false>;
     cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), Gm::THREADS, Gm::SMEM, p.num_tiles, &grid);
@@ -607,8 +610,7 @@ static cudaError_t launch_r2c_big(FftParams p, float* scratch, size_t scratch_by
     const long long fit = (long long)(scratch_bytes / Gm::SCRATCH_PER_CTA);
     if (fit < 1) return cudaErrorInvalidValue;
     if (grid > fit) grid = (int)fit;
-    kern<<<grid, Gm::THREADS, Gm::SMEM, st>>>(tm, tmny, p, reinterpret_cast<float2*>(scratch));
-    return cudaGetLastError();
+    return dep_launch(false, kern, dim3(grid), dim3(Gm::THREADS), Gm::SMEM, st, tm, tmny, p, reinterpret_cast<float2*>(scratch));
     }
 }
 
@@ -627,8 +629,7 @@ static cudaError_t launch_c2r_big(FftParams p, float* scratch, size_t scratch_by
         auto kern = c2r_big_kernel<N, true>;
         cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), Gm::THREADS, Gm::SMEM_SS, p.num_tiles, &grid);
         if (e != cudaSuccess) return e;
-        kern<<<grid, Gm::THREADS, Gm::SMEM_SS, st>>>(tm, tmny, p, nullptr);
-        return cudaGetLastError();
+        return dep_launch(false, kern, dim3(grid), dim3(Gm::THREADS), Gm::SMEM_SS, st, tm, tmny, p, (float2*)nullptr);
     } else {
     auto kern = c2r_big_kernel<N, false>;
     constexpr size_t SMEM = Gm::SMEM;
@@ -637,8 +638,7 @@ static cudaError_t launch_c2r_big(FftParams p, float* scratch, size_t scratch_by
     const long long fit = (long long)(scratch_bytes / Gm::SCRATCH_PER_CTA);
     if (fit < 1) return cudaErrorInvalidValue;
     if (grid > fit) grid = (int)fit;
-    kern<<<grid, Gm::THREADS, SMEM, st>>>(tm, tmny, p, reinterpret_cast<float2*>(scratch));
-    return cudaGetLastError();
+    return dep_launch(false, kern, dim3(grid), dim3(Gm::THREADS), SMEM, st, tm, tmny, p, reinterpret_cast<float2*>(scratch));
     }
 }
 

@@ -47,6 +47,7 @@
 
 #include "fft_core.cuh"
 #include "tma_util.cuh"
+#include "dep_launch.cuh"
 
 namespace fc {
 
@@ -77,6 +78,7 @@ struct FftParams {
     int nty, ntx;
     int step_y, step_x;
     int oy, ox;
+    int overlap;            // host only: launch as a programmatic dependent of the previous kernel
 };
 
 // Geometry of the half-spectrum scratch ("mid") of one plane in shared memory:
@@ -297,11 +299,13 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
         tcol = t - row * tpr;
     };
 
+    dep_trigger();
     if (tid == 0) {
         fk_mbar_init(bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    dep_wait();                     // no global access above this line
 
     // Side jobs are spread over different warps so that no single thread strings them
     // together: thread T/2 issues the input copy, the last warp issues the TMA stores.
@@ -724,6 +728,7 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
     auto fetch_tile = [&](int row, int tcol) { fetch_into(row, tcol, sStage, bar); };
     uint32_t phase = 0;             // DB: bit b is the phase of buffer b's barrier
     int row = blockIdx.x / tpr, tcol = blockIdx.x - (blockIdx.x / tpr) * tpr;
+    dep_trigger();
     if constexpr (TMA) {
         if (tid == 0) {
             fk_mbar_init(bar0, 1);
@@ -731,6 +736,7 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
         __syncthreads();
+        dep_wait();                 // no global access above this line
         if (is_fetcher && blockIdx.x < p.num_tiles) fetch_tile(row, tcol);
         if constexpr (DB) {
             if (is_fetcher && blockIdx.x + gridDim.x < p.num_tiles) {
@@ -739,6 +745,8 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
                 fetch_into(r1, c1, sStage0 + STAGE_FLOATS, bar0 + 8u);
             }
         }
+    } else {
+        dep_wait();
     }
     int buf = 0;
 
@@ -1048,8 +1056,7 @@ static cudaError_t launch_r2c_n(FftParams pa, const FftParams* pb_in, cudaStream
     cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), N * G, smem,
                                     (long long)pa.num_tiles + pb.num_tiles, &grid);
     if (e != cudaSuccess) return e;
-    kern<<<grid, N * G, smem, st>>>(tma, tmb, pa, pb);
-    return cudaGetLastError();
+    return dep_launch(false, kern, dim3(grid), dim3(N * G), smem, st, tma, tmb, pa, pb);
 }
 
 // Plane sizes whose inverse transform double-buffers its staging tile.
@@ -1078,8 +1085,7 @@ static cudaError_t launch_c2r_n(FftParams p, cudaStream_t st) {
     int grid = 0;
     cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), N * G, smem, p.num_tiles, &grid);
     if (e != cudaSuccess) return e;
-    kern<<<grid, N * G, smem, st>>>(tm, p);
-    return cudaGetLastError();
+    return dep_launch(p.overlap != 0, kern, dim3(grid), dim3(N * G), smem, st, tm, p);
 }
 
 template <bool FREQ>

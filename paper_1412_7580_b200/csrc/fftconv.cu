@@ -276,8 +276,13 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     gp.lda = d.a.spec.ld; gp.ldb = d.b.spec.ld; gp.ldc = d.c.spec.ld;
     gp.transA = d.transA; gp.transB = d.transB; gp.conjA = d.conjA; gp.conjB = d.conjB;
     g_launches.fetch_add(1, std::memory_order_relaxed);
+    // the kernels of a pass overlap their ramp-up with the predecessor's drain where that
+    // was measured to pay (see dep_launch.cuh)
+    const bool tensor = resolve_math(*plan, d) == FFTCONV_MATH_TF32;
+    const bool overlap = !big && !timing && (tensor || plan->n >= 32);
+    gp.overlap = (overlap && (need_a || need_b)) ? 1 : 0;       // predecessor: this pass's forward transforms
     cudaError_t ge;
-    if (resolve_math(*plan, d) == FFTCONV_MATH_TF32) ge = fc::launch_cgemm_tc(gp, status, st);
+    if (tensor) ge = fc::launch_cgemm_tc(gp, status, st);
     else ge = fc::launch_cgemm_ffma(gp, st);
     if (ge != cudaSuccess) return FFTCONV_ECUDA;
     mark(3);
@@ -290,6 +295,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     ip.step_y = d.c.step_y; ip.step_x = d.c.step_x; ip.oy = d.c.oy; ip.ox = d.c.ox;
     ip.scale = 1.0f / ((float)plan->n * (float)plan->n);
     ip.accumulate = accumulate ? 1 : 0;
+    ip.overlap = overlap ? 1 : 0;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if ((big ? fc::launch_c2r_two_pass(plan->n, ip, scratch, scratch_bytes, st)
              : fc::launch_c2r<true>(plan->n, ip, st)) != cudaSuccess)

@@ -165,3 +165,43 @@ def test_sweep_subset():
         cw = wl.sample_coords(dw.shape, 60, seed=s.point + 2)
         assert relerr(dw[cw[:, 0], cw[:, 1], cw[:, 2], cw[:, 3]],
                       oracle.accgrad_at(dy, x, s.kh, s.kw, cw)) <= TOL[eff[2]], s
+
+
+@pytest.mark.parametrize("dims", [(6, 20, 24, 16, 16, 3, 3, 16), (4, 24, 40, 31, 31, 5, 5, 32),
+                                  (2, 40, 36, 64, 64, 7, 7, 64)])
+def test_steps_back_to_back_without_synchronisation(dims):
+    """Kernels of consecutive passes overlap their ramp-up with the predecessor's drain.  Every
+    pass reuses the same workspace, so a kernel that started reading or writing too early would
+    corrupt a neighbour's spectra: several steps on changing inputs with no host synchronisation
+    in between, every step's outputs checked afterwards."""
+    import torch
+    import oracle
+    import paper_1412_7580_b200 as fc
+    from paper_1412_7580_b200 import workloads as wl
+    s = wl.ConvShape("b2b", *dims, cfg=8, point=sum(dims))
+    p = fc.conv_plan(*s.args())
+    fc.conv_plan_set_math(p, fc.MATH_TF32)
+    fc.conv_plan_alloc_workspace(p)
+    steps = 4
+    ins, outs = [], []
+    for i in range(steps):
+        si = wl.ConvShape("b2b", *dims, cfg=8, point=sum(dims) + 100 * i)
+        x, w, dy = wl.make_x(si), wl.make_w(si), wl.make_dy(si)
+        ins.append((x, w, dy))
+        outs.append((torch.empty((s.S, s.fp, s.oh, s.ow), device="cuda"),
+                     torch.empty((s.S, s.f, s.h, s.w), device="cuda"),
+                     torch.empty((s.fp, s.f, s.kh, s.kw), device="cuda")))
+    dev = [tuple(torch.from_numpy(a).cuda() for a in t) for t in ins]
+    torch.cuda.synchronize()
+    for (xd, wd, dyd), (y, dx, dw) in zip(dev, outs):
+        fc.conv_fprop(p, xd, wd, y)
+        fc.conv_bprop(p, dyd, wd, dx)
+        fc.conv_accgrad(p, dyd, xd, dw)
+    torch.cuda.synchronize()
+    assert fc.conv_plan_status(p) == 0
+    eff = [fc.conv_plan_pass_math(p, k) for k in range(3)]
+    for (x, w, dy), (y, dx, dw) in zip(ins, outs):
+        assert relerr(y.cpu().numpy().astype(np.float64), oracle.fprop(x, w)) <= TOL[eff[0]]
+        assert relerr(dx.cpu().numpy().astype(np.float64), oracle.bprop(dy, w, s.h, s.w)) <= TOL[eff[1]]
+        assert relerr(dw.cpu().numpy().astype(np.float64), oracle.accgrad(dy, x, s.kh, s.kw)) <= TOL[eff[2]]
+    fc.conv_plan_destroy(p)
