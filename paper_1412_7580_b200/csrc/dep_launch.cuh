@@ -45,8 +45,9 @@ static bool dep_launch_enabled() {
 //  * the forward transforms as dependents of the previous pass's inverse transform gain
 //    nothing at n <= 32, and at n = 64 a training step took 1.14 ms instead of 0.74;
 //  * the two-pass transforms (n = 128) lose 2-6 % per pass as dependents or as predecessors;
-//  * the FFMA contraction at n <= 16 loses up to 12 % (its small CTAs share SMs with the
-//    waiting CTAs of the inverse transform).
+//  * the FFMA contraction at n <= 16 with a long reduction (K > 64) loses up to 12 % (its
+//    small CTAs share SMs with the waiting CTAs of the inverse transform); with K <= 64 the
+//    passes are shorter (24 -> 21 us on an S8 f4 f'8 16 x 16 layer).
 // The callers set the flag accordingly; everything else is launched the plain way.
 template <typename... KArgs, typename... Args>
 static cudaError_t dep_launch(bool overlap, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,

@@ -279,7 +279,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     // the kernels of a pass overlap their ramp-up with the predecessor's drain where that
     // was measured to pay (see dep_launch.cuh)
     const bool tensor = resolve_math(*plan, d) == FFTCONV_MATH_TF32;
-    const bool overlap = !big && !timing && (tensor || plan->n >= 32);
+    const bool overlap = !big && !timing && (tensor || plan->n >= 32 || d.K <= 64);
     gp.overlap = (overlap && (need_a || need_b)) ? 1 : 0;       // predecessor: this pass's forward transforms
     cudaError_t ge;
     if (tensor) ge = fc::launch_cgemm_tc(gp, status, st);
