@@ -44,7 +44,8 @@ static bool dep_launch_enabled() {
 //    1-7 % shorter passes at n <= 64 with the tensor-core contraction;
 //  * the forward transforms as dependents of the previous pass's inverse transform gain
 //    nothing at n <= 32, and at n = 64 a training step took 1.14 ms instead of 0.74;
-//  * the two-pass transforms (n = 128) lose 2-6 % per pass as dependents or as predecessors;
+//  * with the two-pass transforms (n = 128) a pass is 0.5 % longer with the contraction as a
+//    dependent and 2.5 % longer with the inverse transform as one (2-6 % over the sweep);
 //  * the FFMA contraction at n <= 16 with a long reduction (K > 64) loses up to 12 % (its
 //    small CTAs share SMs with the waiting CTAs of the inverse transform); with K <= 64 the
 //    passes are shorter (24 -> 21 us on an S8 f4 f'8 16 x 16 layer).
