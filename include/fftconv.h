@@ -82,7 +82,8 @@ int conv_plan_pass_math(const conv_plan_t* plan, int pass);
  * the two operands and of the result (Section 6 lists the same buffers), in the
  * plan's private frequency-major layout; plans with n = 128 add the scratch
  * that the transforms of large planes pass their half spectra through between
- * the two 1-D passes (80 MiB).  0 on a null plan. */
+ * the two 1-D passes (80 MiB = 83.9e6 bytes: 512 KiB for each of up to 160
+ * resident CTAs).  0 on a null plan. */
 size_t conv_plan_workspace_bytes(const conv_plan_t* plan);
 
 /* Lend the plan `bytes` of device memory at `dev_ptr` (256-byte aligned).  The
@@ -119,7 +120,9 @@ int conv_fprop(conv_plan_t* plan, const float* x, const float* w, float* y, void
  *    (different streams, no dependency) race on the array: serialise them.
  *  - A bounded device-side wait that runs out is recorded in the array's header,
  *    which no entry point reads back; use conv_fprop + conv_plan_status where
- *    that diagnosis matters. */
+ *    that diagnosis matters.
+ *  - The first calls on a device may come from several host threads at once:
+ *    they all look up and store the same address. */
 #define FFTCONV_NOALLOC_BYTES (32u << 20)
 int conv_fprop_noalloc(conv_plan_t* plan, const float* x, const float* w, float* y,
                        void* cuda_stream);
@@ -180,8 +183,21 @@ int conv_plan_tile_basis(const conv_plan_t* plan);
 
 /* Reads the plan's device status word (synchronises the device).  FFTCONV_OK,
  * or FFTCONV_EDEVICE_TIMEOUT if a bounded wait inside a kernel gave up since
- * the last call (the word is then cleared), or ECUDA. */
+ * the last call (the word is then cleared), or ECUDA.  Every kernel of a pass
+ * -- the forward and inverse transforms and the tensor-core contraction --
+ * bounds each wait on an asynchronous copy or on the tensor cores; when a limit
+ * runs out the kernel raises this word, lets the copies and MMAs it has issued
+ * finish (again bounded), frees its tensor memory and returns, so the context
+ * stays usable.  The results of such a pass are unspecified. */
 int conv_plan_status(conv_plan_t* plan);
+
+/* Limit of one bounded device-side wait, in SM clock cycles; 0 restores the
+ * default (2e9 cycles, about a second).  A diagnostic hook: a limit shorter
+ * than a copy's normal latency makes the waits run out on purpose, which is how
+ * the tests exercise the give-up paths without hanging anything (the draining
+ * waits after a give-up always keep the default limit).  EINVAL: null plan or a
+ * negative limit. */
+int conv_plan_set_wait_limit(conv_plan_t* plan, long long sm_cycles);
 
 /* Frees the plan (host memory and its timing events; never the workspace). */
 int conv_plan_destroy(conv_plan_t* plan);

@@ -23,6 +23,7 @@ EXPORTS = (
     "conv_plan_set_workspace", "conv_plan_set_spectrum_reuse", "conv_plan_invalidate_spectra",
     "conv_plan_set_tiling", "conv_plan_tile_basis",
     "conv_fprop", "conv_fprop_noalloc", "conv_bprop", "conv_accgrad", "conv_plan_status",
+    "conv_plan_set_wait_limit",
     "conv_plan_destroy", "conv_plan_enable_stage_timing", "conv_plan_stage_times_ms", "fft2d_r2c", "fft2d_c2r", "fft1d_r2c", "fft1d_c2r", "fftconv_bin_contract",
     "fftconv_status_string", "fftconv_launch_count",
 )
@@ -62,6 +63,7 @@ def lib():
         L.conv_bprop.argtypes = [p, p, p, p, p]
         L.conv_accgrad.argtypes = [p, p, p, p, i, p]
         L.conv_plan_status.argtypes = [p]
+        L.conv_plan_set_wait_limit.argtypes = [p, ctypes.c_longlong]
         L.conv_plan_destroy.argtypes = [p]
         L.conv_plan_enable_stage_timing.argtypes = [p, i]
         L.conv_plan_stage_times_ms.argtypes = [p, p]
@@ -244,6 +246,11 @@ def conv_accgrad(plan: Plan, dy, x, dw, accumulate=False, stream=None) -> None:
 
 def conv_plan_status(plan: Plan) -> int:
     return int(lib().conv_plan_status(plan.handle))
+
+
+def conv_plan_set_wait_limit(plan: Plan, sm_cycles: int) -> None:
+    """Limit of one bounded device-side wait in SM cycles (0 = default, about a second)."""
+    _check(lib().conv_plan_set_wait_limit(plan.handle, int(sm_cycles)), "conv_plan_set_wait_limit")
 
 
 def conv_plan_enable_stage_timing(plan: Plan, enable=1) -> None:

@@ -27,6 +27,7 @@ struct GemmParams {
     int transA, transB;   // operand stored [K][rows] instead of [rows][K]
     int conjA, conjB;     // use the complex conjugate of the operand
     int overlap;          // host only: launch as a programmatic dependent of the previous kernel
+    long long wait_cycles; // host only: limit of a bounded wait in the tensor-core kernel (<= 0: default)
 };
 
 constexpr int FG_BM = 64, FG_BN = 64, FG_BK = 16, FG_PAD = 4, FG_T = 256;
@@ -38,8 +39,11 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
     dep_trigger();
     dep_wait();                     // no global access above this line
     const int tid = threadIdx.x;
-    const int bin = blockIdx.z;
-    const int m_blk = blockIdx.y * FG_BM, n_blk = blockIdx.x * FG_BN;
+    // grid: x = (row block, column block) linearised (tiled plans can have millions of row
+    // blocks, more than grid.y takes), y = bin
+    const int bin = blockIdx.y;
+    const int n_blocks = (p.N + FG_BN - 1) / FG_BN;
+    const int m_blk = (int)(blockIdx.x / n_blocks) * FG_BM, n_blk = (int)(blockIdx.x % n_blocks) * FG_BN;
     const size_t planeA = (size_t)(p.transA ? p.K : p.M) * p.lda,
                  planeB = (size_t)(p.transB ? p.K : p.N) * p.ldb, planeC = (size_t)p.M * p.ldc;
     const float sa = p.conjA ? -1.0f : 1.0f, sb = p.conjB ? -1.0f : 1.0f;
@@ -154,8 +158,9 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
 }
 
 static cudaError_t launch_cgemm_ffma(const GemmParams& p, cudaStream_t st) {
-    dim3 grid((p.N + FG_BN - 1) / FG_BN, (p.M + FG_BM - 1) / FG_BM, p.bins);
-    if (grid.y > 65535u || grid.z > 65535u) return cudaErrorInvalidValue;
+    const long long blocks = (long long)((p.N + FG_BN - 1) / FG_BN) * ((p.M + FG_BM - 1) / FG_BM);
+    if (blocks > 0x7fffffffLL || p.bins > 65535) return cudaErrorInvalidValue;
+    dim3 grid((unsigned)blocks, (unsigned)p.bins, 1);
     return dep_launch(p.overlap != 0, cgemm_ffma_kernel, grid, dim3(FG_T), 0, st, p);
 }
 

@@ -34,9 +34,12 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "cgemm_ffma.cuh"
 #include "tma_util.cuh"
 #include "dep_launch.cuh"
+#include "fft_kernels.cuh"
 
 namespace fc {
 
@@ -55,6 +58,7 @@ struct TcParams {
     int m_tiles, n_tiles, k_blocks;
     int conjA, conjB;
     int* status;
+    long long wait_cycles;      // limit of one wait in SM clock cycles (the draining waits keep TC_WAIT_CYCLES)
 };
 
 static inline bool tc_shape_supported(int M, int N, int K) {
@@ -94,15 +98,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait: false when the limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
+// Bounded wait: false when the limit ran out or another role already gave up.  The first
+// probe does not block; before every further (possibly suspending) attempt the clock and
+// the abort flag are checked.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          long long limit) {
+    if (fk_mbar_test_wait(bar, parity)) return true;
     const long long t0 = clock64();
     for (;;) {
-        for (int i = 0; i < 256; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > TC_WAIT_CYCLES) return false;
+        if (clock64() - t0 > limit) return false;
+        if (mbar_try_wait(bar, parity)) return true;
     }
 }
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
@@ -239,7 +245,7 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % TC_STAGES;
                     const uint32_t ph = (uint32_t)(it / TC_STAGES) & 1u;
-                    if (!mbar_wait(empty(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(empty(s), ph ^ 1u, abort_flag, p.wait_cycles)) { ok = false; break; }
                     const uint32_t dst = tiles + s * TC_STAGE_BYTES;
                     mbar_expect_tx(full(s), TC_STAGE_BYTES);
 #pragma unroll
@@ -289,13 +295,13 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             bool ok = true;
             for (int t = blockIdx.x; ok && t < num_tiles; t += gridDim.x, ++tl) {
                 const int buf = tl & 1;
-                if (!mbar_wait(tempty(buf), ((uint32_t)(tl >> 1) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(tempty(buf), ((uint32_t)(tl >> 1) & 1u) ^ 1u, abort_flag, p.wait_cycles)) { ok = false; break; }
                 tc_fence_after_sync();
                 const uint32_t d_re = tmem_base + (uint32_t)buf * 256u;
                 const uint32_t d_im = d_re + 128u;
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % TC_STAGES;
-                    if (!mbar_wait(full(s), (uint32_t)(it / TC_STAGES) & 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(full(s), (uint32_t)(it / TC_STAGES) & 1u, abort_flag, p.wait_cycles)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t src = tiles + s * TC_STAGE_BYTES;
                     const uint64_t a_re = TA ? tc_smem_desc_mn(src) : tc_smem_desc(src);
@@ -340,7 +346,7 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int m_t = (t / p.n_tiles) % p.m_tiles;
             const int bin = t / (p.n_tiles * p.m_tiles);
             const int buf = tl & 1;
-            if (!mbar_wait(tfull(buf), (uint32_t)(tl >> 1) & 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(tfull(buf), (uint32_t)(tl >> 1) & 1u, abort_flag, p.wait_cycles)) { ok = false; break; }
             tc_fence_after_sync();
             const int row0 = m_t * TC_BM + q * 32;
             const int col0 = n_t * TC_BN;
@@ -397,14 +403,14 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 template <bool TA, bool TB>
 static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStream_t st, int sm_count) {
     auto kern = cgemm_tc_kernel<TA, TB>;
-    static unsigned long long attr_set_devices = 0;     // one bit per device ordinal
+    static std::atomic<unsigned long long> attr_set_devices{0};     // one bit per device ordinal
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
-    if (dev >= 64 || !((attr_set_devices >> dev) & 1ull)) {
+    if (dev < 0 || dev >= 64 || !((attr_set_devices.load(std::memory_order_acquire) >> dev) & 1ull)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)TC_SMEM_BYTES);
         if (e != cudaSuccess) return e;
-        if (dev < 64) attr_set_devices |= 1ull << dev;
+        if (dev >= 0 && dev < 64) attr_set_devices.fetch_or(1ull << dev, std::memory_order_release);
     }
     CUtensorMap tmA, tmB, tmC;
     // k-contiguous: rows = M (or N), cols = K, box 32 k x 128 rows;
@@ -424,6 +430,7 @@ static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStrea
     p.k_blocks = (g.K + TC_BK - 1) / TC_BK;
     p.conjA = g.conjA; p.conjB = g.conjB;
     p.status = status;
+    p.wait_cycles = g.wait_cycles > 0 ? g.wait_cycles : TC_WAIT_CYCLES;
     const long long tiles = (long long)p.bins * p.m_tiles * p.n_tiles;
     if (tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
@@ -431,14 +438,8 @@ static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStrea
 }
 
 static cudaError_t launch_cgemm_tc(const GemmParams& g, int* status, cudaStream_t st) {
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-    }
+    const int sm_count = fft_sm_count();        // of the current device
+    if (sm_count < 1) return cudaErrorInvalidDevice;
     if (g.transA) return g.transB ? launch_cgemm_tc_t<true, true>(g, status, st, sm_count)
                                   : launch_cgemm_tc_t<true, false>(g, status, st, sm_count);
     return g.transB ? launch_cgemm_tc_t<false, true>(g, status, st, sm_count)

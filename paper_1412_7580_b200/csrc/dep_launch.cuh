@@ -13,8 +13,6 @@
 #pragma once
 
 #include <cuda_runtime.h>
-#include <stdlib.h>
-
 #include <utility>
 
 namespace fc {
@@ -26,16 +24,6 @@ __device__ __forceinline__ void dep_trigger() {
 // Block until every kernel this launch depends on has completed and flushed its writes.
 __device__ __forceinline__ void dep_wait() {
     asm volatile("griddepcontrol.wait;" ::: "memory");
-}
-
-// FFTCONV_SERIAL_LAUNCH=1 launches every kernel the plain way (for measurements).
-static bool dep_launch_enabled() {
-    static int state = -1;
-    if (state < 0) {
-        const char* e = getenv("FFTCONV_SERIAL_LAUNCH");
-        state = (e && e[0] == '1') ? 0 : 1;
-    }
-    return state == 1;
 }
 
 // `overlap` = false launches the plain way.  Where overlapping pays was measured on B200
@@ -62,7 +50,7 @@ static cudaError_t dep_launch(bool overlap, void (*kern)(KArgs...), dim3 grid, d
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = (overlap && dep_launch_enabled()) ? 1 : 0;
+    cfg.numAttrs = overlap ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 

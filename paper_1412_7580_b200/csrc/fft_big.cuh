@@ -35,8 +35,6 @@
 // the team's buffer, cropped / scaled / accumulated stores).
 #pragma once
 
-#include <stdlib.h>
-
 #include "fft_kernels.cuh"
 
 namespace fc {
@@ -101,97 +99,27 @@ static bool big_make_map(CUtensorMap* map, const float* spec, const FftParams& p
                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// L2 eviction hints (FC_BIG_L2_HINTS=1): "keep" for the scratch, "stream" for planes and
-// spectra.  Measured on B200: DRAM traffic of the forward kernel falls by about 15 %, but the
-// kernels run 5-10 % slower, so the hints are compiled out by default.
-#ifndef FC_BIG_L2_HINTS
-#define FC_BIG_L2_HINTS 0
-#endif
-__device__ __forceinline__ uint64_t big_policy_keep() {
-    uint64_t pol = 0;
-#if FC_BIG_L2_HINTS
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-#endif
-    return pol;
-}
-__device__ __forceinline__ uint64_t big_policy_stream() {
-    uint64_t pol = 0;
-#if FC_BIG_L2_HINTS
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
-#endif
-    return pol;
-}
 __device__ __forceinline__ void fk_tma_store_4d(const CUtensorMap* map, uint32_t src, int c0, int c1,
-                                                int c2, int c3, uint64_t pol) {
-#if FC_BIG_L2_HINTS
-    asm volatile(
-        "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3, %4, %5}], [%1], %6;"
-        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "l"(pol)
-        : "memory");
-#else
-    (void)pol;
+                                                int c2, int c3) {
     asm volatile(
         "cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%2, %3, %4, %5}], [%1];"
         ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
-#endif
 }
 __device__ __forceinline__ void fk_tma_load_4d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
-                                               int c2, int c3, uint32_t bar, uint64_t pol) {
-#if FC_BIG_L2_HINTS
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-        " [%0], [%1, {%3, %4, %5, %6}], [%2], %7;"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
-          "l"(pol)
-        : "memory");
-#else
-    (void)pol;
+                                               int c2, int c3, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes"
         " [%0], [%1, {%3, %4, %5, %6}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
-#endif
 }
-__device__ __forceinline__ void fk_cp16(uint32_t dst, const void* src, uint64_t pol) {
-#if FC_BIG_L2_HINTS
-    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;"
-                 ::"r"(dst), "l"(src), "l"(pol) : "memory");
-#else
-    (void)pol;
+__device__ __forceinline__ void fk_cp16(uint32_t dst, const void* src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-#endif
 }
-__device__ __forceinline__ void big_st2(float2* a, float2 v, uint64_t pol) {
-#if FC_BIG_L2_HINTS
-    asm volatile("st.global.L2::cache_hint.v2.f32 [%0], {%1, %2}, %3;"
-                 ::"l"(a), "f"(v.x), "f"(v.y), "l"(pol) : "memory");
-#else
-    (void)pol;
-    *a = v;
-#endif
-}
-__device__ __forceinline__ void big_st4(float4* a, float4 v, uint64_t pol) {
-#if FC_BIG_L2_HINTS
-    asm volatile("st.global.L2::cache_hint.v4.f32 [%0], {%1, %2, %3, %4}, %5;"
-                 ::"l"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w), "l"(pol) : "memory");
-#else
-    (void)pol;
-    __stcg(a, v);
-#endif
-}
-__device__ __forceinline__ float2 big_ld2(const float2* a, uint64_t pol) {
-#if FC_BIG_L2_HINTS
-    float2 v;
-    asm volatile("ld.global.cg.L2::cache_hint.v2.f32 {%0, %1}, [%2], %3;"
-                 : "=f"(v.x), "=f"(v.y) : "l"(a), "l"(pol) : "memory");
-    return v;
-#else
-    (void)pol;
-    return __ldcg(a);
-#endif
-}
+__device__ __forceinline__ void big_st2(float2* a, float2 v) { *a = v; }
+__device__ __forceinline__ void big_st4(float4* a, float4 v) { __stcg(a, v); }
+__device__ __forceinline__ float2 big_ld2(const float2* a) { return __ldcg(a); }
 template <int TEAM>
 __device__ __forceinline__ void big_team_sync(int team) {
     asm volatile("bar.sync %0, %1;" ::"r"(1 + team), "n"(TEAM) : "memory");
@@ -220,12 +148,6 @@ __device__ __forceinline__ void big_split4_rows(const float2* rowp, float (&ar)[
     });
 }
 
-#ifdef FC_EXP_TIMELINE
-#define BIG_TICK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { long long t_ = clock64(); fc_timeline[i] += t_ - tl_last; tl_last = t_; } } while (0)
-#else
-#define BIG_TICK(i) do { } while (0)
-#endif
-
 // ---------------------------------------------------------------------------
 // Forward.
 // ---------------------------------------------------------------------------
@@ -251,7 +173,6 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
     const int q4 = tid / Gm::ROWS, rB = tid - q4 * Gm::ROWS;   // step B: (quarter, row = ky_local*8 + plane)
     const int h = p.h, w = p.w, hw = h * w;
     const int tpr = p.tiles_per_row;
-    const uint64_t keep = big_policy_keep(), stream = big_policy_stream();
     dep_trigger();
     dep_wait();                     // no global access above this line
 
@@ -261,7 +182,7 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
         float* dst = reinterpret_cast<float*>(buf);
         if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
             const int vec = hw >> 2;
-            for (int i = tid; i < vec; i += T) fk_cp16(fk_smem_u32(dst + 4 * i), src + 4 * i, stream);
+            for (int i = tid; i < vec; i += T) fk_cp16(fk_smem_u32(dst + 4 * i), src + 4 * i);
             for (int i = 4 * vec + tid; i < hw; i += T) dst[i] = __ldg(src + i);
         } else {
             for (int i = tid; i < hw; i += T) dst[i] = __ldg(src + i);
@@ -275,15 +196,12 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
         for (int i = tid; i < Gm::ROWS * PER_ROW; i += T) {
             const int rr = i / PER_ROW, pc = i - rr * PER_ROW;
             const int g = rr & (G - 1), ky = ci * KC + (rr >> 3);
-            fk_cp16(fk_smem_u32(dst + rr * PITCH + 2 * pc), scratch + ((size_t)(g * M + ky) * N + 2 * pc), keep);
+            fk_cp16(fk_smem_u32(dst + rr * PITCH + 2 * pc), scratch + ((size_t)(g * M + ky) * N + 2 * pc));
         }
     };
 
     bool store_pending = false;
     bool team_store_pending = false;        // SS: the team's last store may still be reading its buffer
-#ifdef FC_EXP_TIMELINE
-    long long tl_last = clock64();
-#endif
     for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x) {
         const int row = tile / tpr, tcol = tile - row * tpr;
         const int c0 = tcol * G;
@@ -297,14 +215,11 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 team_store_pending = false;
             }
         }
-        BIG_TICK(0);
         if (team < gcount) issue_plane(row, c0, team);
         fk_cp_commit();
         for (int g = team; g < gcount; g += NT) {
-            BIG_TICK(1);
             fk_cp_wait<0>();
             big_team_sync<T>(team);                           // plane g has landed for the team
-            BIG_TICK(2);
             const float* pl = reinterpret_cast<const float*>(buf) + cA;
             float ar[H], ai[H];
             const bool live = cA < w;
@@ -316,14 +231,12 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 if (q2 == 0) rfft_half_split<N, 0>(x, ar, ai);
                 else         rfft_half_split<N, 1>(x, ar, ai);
             }
-            BIG_TICK(3);
             big_team_sync<T>(team);                           // plane g is in registers: the buffer takes the next one
             if (g + NT < gcount) issue_plane(row, c0, g + NT);
             fk_cp_commit();
-            BIG_TICK(4);
             float2* dst = scratch + (size_t)g * PS + cA;
             auto put = [&](float2* a, float2 v) {
-                if constexpr (SS) *a = v; else big_st2(a, v, keep);
+                if constexpr (SS) *a = v; else big_st2(a, v);
             };
             if (live) {
                 if (q2 == 0) {
@@ -348,10 +261,8 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 });
             }
         }
-        BIG_TICK(5);
         fk_cp_wait<0>();
         __syncthreads();                                   // the scratch is complete
-        BIG_TICK(6);
 
         // ---- B: row transforms; chunks team, team + NT, .. --------------------------------
         constexpr int CHUNKS = M / KC;
@@ -372,14 +283,12 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
             else if (q4 == 1) big_split4_rows<N, false, 1>(rowp, ar, ai);
             else if (q4 == 2) big_split4_rows<N, false, 2>(rowp, ar, ai);
             else              big_split4_rows<N, false, 3>(rowp, ar, ai);
-            BIG_TICK(7);
             if constexpr (SS) {
                 // the rows were read in place; the team's buffer is still the previous staging
                 // tile until its store has been read out
                 if (tid == 0 && team_store_pending) fk_bulk_wait_read();
             }
             big_team_sync<T>(team);                           // the chunk is in registers: the buffer becomes the staging tile
-            BIG_TICK(8);
             cfft<L, false>(ar, ai);                        // ar/ai[m] = F[kx = 4m + q4]
             float* sStage = reinterpret_cast<float*>(buf);
             float* o = sStage + q4 * Gm::ROWS + rB;
@@ -406,23 +315,19 @@ r2c_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                     b[kp * G] = xnr; b[(N + kp) * G] = -xni;
                 }
             }
-            BIG_TICK(9);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             big_team_sync<T>(team);
-            BIG_TICK(10);
             if (tid == 0) {
-                fk_tma_store_4d(&tmS, fk_smem_u32(sStage), c0, row, ci * KC, 0, stream);
-                if (ci == 0) fk_tma_store_4d(&tmNy, fk_smem_u32(sNy), c0, row, M, 0, stream);
+                fk_tma_store_4d(&tmS, fk_smem_u32(sStage), c0, row, ci * KC, 0);
+                if (ci == 0) fk_tma_store_4d(&tmNy, fk_smem_u32(sNy), c0, row, M, 0);
                 fk_bulk_commit();
                 if constexpr (!SS) fk_bulk_wait_read();    // the buffer may be overwritten after this
             }
             store_pending = true;
             team_store_pending = true;
             if constexpr (!SS) big_team_sync<T>(team);
-            BIG_TICK(11);
         }
         __syncthreads();                                   // both teams are done with the scratch
-        BIG_TICK(12);
     }
     if (tid == 0 && store_pending) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
@@ -455,7 +360,6 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
     const float scale = p.scale;
     const bool acc = p.accumulate != 0;
     constexpr int CHUNKS = M / KC;
-    const uint64_t keep = big_policy_keep(), stream = big_policy_stream();
 
     dep_trigger();
     if (tid == 0) {
@@ -476,10 +380,10 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
         for (int ci = team; ci < CHUNKS; ci += NT) {
             if (tid == 0) {
                 fk_mbar_expect_tx(bar, (uint32_t)(Gm::STAGE + (ci == 0 ? Gm::STAGE_NY : 0)));
-                fk_tma_load_4d(fk_smem_u32(buf), &tmS, c0, row, ci * KC, 0, bar, stream);
-                if (ci == 0) fk_tma_load_4d(fk_smem_u32(sNy), &tmNy, c0, row, M, 0, bar, stream);
+                fk_tma_load_4d(fk_smem_u32(buf), &tmS, c0, row, ci * KC, 0, bar);
+                if (ci == 0) fk_tma_load_4d(fk_smem_u32(sNy), &tmNy, c0, row, M, 0, bar);
             }
-            if (!dead && !fk_mbar_wait(bar, phase)) dead = true;
+            if (!dead && !fk_wait_or_report(bar, phase, p.wait_cycles, p.status)) dead = true;
             phase ^= 1u;
             float* st = reinterpret_cast<float*>(buf);
             if (ci == 0) {
@@ -528,7 +432,7 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
                 const int rr = i / PER_ROW, pc = i - rr * PER_ROW;
                 const int g = rr & (G - 1), ky = ci * KC + (rr >> 3);
                 const float4 v = *reinterpret_cast<const float4*>(sRows + rr * PITCH + 2 * pc);
-                big_st4(reinterpret_cast<float4*>(scratch + ((size_t)(g * M + ky) * N + 2 * pc)), v, keep);
+                big_st4(reinterpret_cast<float4*>(scratch + ((size_t)(g * M + ky) * N + 2 * pc)), v);
             }
             big_team_sync<T>(team);                           // the buffer is free for the next chunk
             }
@@ -543,7 +447,7 @@ c2r_big_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ 
             auto X = [&](auto K) -> float2 {
                 constexpr int k = decltype(K)::value;
                 if constexpr (SS) return src[(size_t)k * RS];
-                else return big_ld2(src + (size_t)k * N, keep);
+                else return big_ld2(src + (size_t)k * N);
             };
             if (q2 == 0) irfft_half<N, 0>(X, er, ei);
             else         irfft_half<N, 1>(X, er, ei);
@@ -642,18 +546,9 @@ static cudaError_t launch_c2r_big(FftParams p, float* scratch, size_t scratch_by
     }
 }
 
-// Which plane sizes take the two-pass kernels.  n = 64 can run on either family; the
-// environment variable FFTCONV_TWO_PASS_64 (0 / 1) overrides the default for measurements.
-static inline bool big_uses_two_pass(int n) {
-    if (n == 128) return true;
-    if (n != 64) return false;
-    static int on = -1;
-    if (on < 0) {
-        const char* e = getenv("FFTCONV_TWO_PASS_64");
-        on = e ? (atoi(e) != 0) : 0;
-    }
-    return on == 1;
-}
+// Which plane sizes take the two-pass kernels.  (They are also instantiated for n = 64, with
+// the scratch in shared memory; measured slower there than the one-pass kernels, so not used.)
+static inline bool big_uses_two_pass(int n) { return n == 128; }
 static cudaError_t launch_r2c_two_pass(int n, const FftParams& p, float* scratch, size_t bytes, cudaStream_t st) {
     return n == 128 ? launch_r2c_big<128>(p, scratch, bytes, st) : launch_r2c_big<64>(p, scratch, bytes, st);
 }

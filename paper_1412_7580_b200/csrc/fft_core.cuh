@@ -111,9 +111,6 @@ FC_HD void cfft(float (&re)[N], float (&im)[N]) {
     if constexpr (N == 1) {
         return;
     } else {
-#ifdef FC_EXP_NOMATH
-        return;     // measurement builds: data movement only (results are wrong)
-#endif
         constexpr int BITS = ilog2(N);
         float br[N], bi[N];
         static_for<N>([&](auto I) {
@@ -171,11 +168,6 @@ FC_HD void cfft(float (&re)[N], float (&im)[N]) {
 template <int N>
 FC_HD void rfft(const float (&x)[N], float (&Xr)[N / 2 + 1], float (&Xi)[N / 2 + 1]) {
     constexpr int M = N / 2;
-#ifdef FC_EXP_NOMATH
-    static_for<M>([&](auto J) { constexpr int j = decltype(J)::value; Xr[j] = x[2 * j]; Xi[j] = x[2 * j + 1]; });
-    Xr[M] = x[0]; Xi[M] = x[1];
-    return;
-#endif
     float zr[M], zi[M];
     static_for<M>([&](auto J) {
         constexpr int j = decltype(J)::value;
@@ -217,11 +209,6 @@ FC_HD void rfft(const float (&x)[N], float (&Xr)[N / 2 + 1], float (&Xi)[N / 2 +
 template <int N>
 FC_HD void irfft(const float (&Xr)[N / 2 + 1], const float (&Xi)[N / 2 + 1], float (&x)[N]) {
     constexpr int M = N / 2;
-#ifdef FC_EXP_NOMATH
-    static_for<M>([&](auto J) { constexpr int j = decltype(J)::value; x[2 * j] = Xr[j]; x[2 * j + 1] = Xi[j]; });
-    x[0] += Xr[M];
-    return;
-#endif
     float zr[M], zi[M];
     zr[0] = Xr[0] + Xr[M];
     zi[0] = Xr[0] - Xr[M];

@@ -43,6 +43,7 @@
 #include <stdint.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "fft_core.cuh"
@@ -79,6 +80,8 @@ struct FftParams {
     int step_y, step_x;
     int oy, ox;
     int overlap;            // host only: launch as a programmatic dependent of the previous kernel
+    int* status;            // device status word raised when a bounded wait runs out (may be null)
+    long long wait_cycles;  // limit of one wait in SM clock cycles; <= 0 selects FK_WAIT_CYCLES
 };
 
 // Geometry of the half-spectrum scratch ("mid") of one plane in shared memory:
@@ -125,15 +128,38 @@ __device__ __forceinline__ bool fk_mbar_try_wait(uint32_t bar, uint32_t parity) 
         : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
     return ok != 0;
 }
-// Bounded wait (about a second); returns false when it ran out.
-__device__ __forceinline__ bool fk_mbar_wait(uint32_t bar, uint32_t parity) {
-    if (fk_mbar_try_wait(bar, parity)) return true;
+__device__ __forceinline__ bool fk_mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Every wait on an mbarrier is bounded: about a second by default, or the limit the plan
+// was given.  Returns false when the limit ran out.  The first probe does not block;
+// try_wait may suspend the thread for a hardware-defined time, so the clock is read before
+// every further attempt and a very short limit really is short.
+constexpr long long FK_WAIT_CYCLES = 2000000000LL;
+__device__ __forceinline__ bool fk_mbar_wait(uint32_t bar, uint32_t parity, long long limit) {
+    if (fk_mbar_test_wait(bar, parity)) return true;
+    if (limit <= 0) limit = FK_WAIT_CYCLES;
     const long long t0 = clock64();
     for (;;) {
-        for (int i = 0; i < 64; ++i)
-            if (fk_mbar_try_wait(bar, parity)) return true;
-        if (clock64() - t0 > 2000000000LL) return false;
+        if (clock64() - t0 > limit) return false;
+        if (fk_mbar_try_wait(bar, parity)) return true;
     }
+}
+// A wait that reports: when the plan's limit runs out the status word is raised, and the copy
+// is then given the full default limit to land -- it must not arrive in shared memory that
+// already belongs to another CTA.  True if the data is there (possibly late, status raised),
+// false if it never came: the caller then leaves its remaining tiles undone and returns.
+__device__ __forceinline__ bool fk_wait_or_report(uint32_t bar, uint32_t parity, long long limit,
+                                                  int* status) {
+    if (fk_mbar_wait(bar, parity, limit)) return true;
+    if (status) atomicExch(status, 1);
+    return fk_mbar_wait(bar, parity, FK_WAIT_CYCLES);
 }
 __device__ __forceinline__ void fk_bulk_g2s(uint32_t dst, const void* src, uint32_t bytes,
                                             uint32_t bar) {
@@ -215,19 +241,6 @@ __device__ __forceinline__ void load_split_narrow(Load&& load, int live, float (
         }
     });
 }
-
-// Measurement builds (never the shipped library; results are wrong or partial):
-//   -DFC_EXP_TIMELINE  cycle counts per phase of the forward tile loops (CTA 0, thread 0), read
-//                      back through fftconv_debug_timeline (exported by such builds only);
-//   -DFC_EXP_NOMATH    (fft_core.cuh) the butterflies are skipped: data movement only;
-//   -DFC_EXP_TMAONLY   the TMA-staged kernels only move their tiles (input copy, spectrum
-//                      tile load / store), no shared-memory passes and no arithmetic.
-#ifdef FC_EXP_TIMELINE
-__device__ long long fc_timeline[16];
-#define FC_TICK(i) do { if (blockIdx.x == 0 && threadIdx.x == 0) { long long t_ = clock64(); fc_timeline[i] += t_ - tl_last; tl_last = t_; } } while (0)
-#else
-#define FC_TICK(i) do { } while (0)
-#endif
 
 // ---------------------------------------------------------------------------
 // Forward: real planes -> half spectra.
@@ -387,9 +400,6 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
     }
     __syncthreads();           // plain-load parts of the first tile are visible to everyone
 
-#ifdef FC_EXP_TIMELINE
-    long long tl_last = clock64();
-#endif
     for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
         if (second_n != second) select(second_n);       // divisions only when the operand changes
         second = second_n; row = row_n; tcol = tcol_n;
@@ -407,9 +417,12 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             }
         }
 
-        FC_TICK(0);
         if (pending) {
-            if (!fk_mbar_wait(bar, phase)) return;     // copy never landed: give up
+            if (!fk_wait_or_report(bar, phase, p0.wait_cycles, p0.status)) {
+                // the copy never landed: let the stores already issued finish and leave
+                if (TMA && store_pending && is_storer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+                return;
+            }
             phase ^= 1u;
         }
         if (WIN && win_pending) {
@@ -417,21 +430,6 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             __syncthreads();
             win_pending = false;
         }
-        FC_TICK(1);
-#ifdef FC_EXP_TMAONLY
-        if (TMA) {
-            if (store_pending && is_storer) fk_bulk_wait_read();
-            __syncthreads();
-            pending = (next < total_tiles) ? stage(second_n, row_n, tcol_n) : false;
-            if (is_storer) {
-                const int b0 = (tid & 31) * D;
-                fk_tma_store_3d(tmS, fk_smem_u32(sStage + (size_t)b0 * G), c0, row, b0);
-                fk_bulk_commit();
-            }
-            store_pending = true;
-            continue;
-        }
-#endif
 
         // 2. column transforms.  Wide planes: thread = (plane gA, column cA), cA < w, one real
         //    FFT of length N each.  Narrow planes (filters): four threads per column, thread
@@ -503,11 +501,8 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
                     cfft<L, false>(br, bi);             // br/bi[k] = X[ky = 4k + q4]
                 }
             }
-            FC_TICK(2);
             if (TMA && store_pending && is_storer) fk_bulk_wait_read();  // staging tile free again
-            FC_TICK(3);
             __syncthreads();   // tile consumed (and the previous tile's step 3 is done with sMid)
-            FC_TICK(4);
             if (!ALIAS) pending = (next < total_tiles) ? stage(second_n, row_n, tcol_n) : false;
             // Rows ky = 0 and ky = N/2 of a real column transform are real: they share the
             // scratch row 0 as (re, im) and are transformed together in step 3.
@@ -538,9 +533,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
                 });
             }
         }
-        FC_TICK(5);
         __syncthreads();
-        FC_TICK(6);
 
         // 3. row transforms: thread = (half q, row kyp, plane gB)
         if (TMA || gB < gcount) {
@@ -557,11 +550,8 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
                 if (q == 0) load_split<N, false, 0>(load, ar, ai);
                 else        load_split<N, false, 1>(load, ar, ai);
             }
-            FC_TICK(7);
             if constexpr (TMA && SALIAS) __syncthreads();   // scratch consumed: it becomes the staging tile
-            FC_TICK(8);
             cfft<M, false>(ar, ai);                     // ar/ai[k] = F[kx = 2k+q]
-            FC_TICK(9);
 
             if constexpr (LAYOUT != LAYOUT_BARE) {
                 // element (part, bin = kx*NC + ky, plane g): staging offset (part*B + bin)*G + g,
@@ -634,7 +624,6 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
                 }
             }
         }
-        FC_TICK(10);
         if constexpr (TMA) {
             // Row ky = 0 of every plane holds Z = FFT(X_0 + i X_{N/2}) of the two real rows:
             // X_0[k] = (Z_k + conj Z_{-k}) / 2,  X_{N/2}[k] = (Z_k - conj Z_{-k}) / (2i); one
@@ -655,9 +644,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            FC_TICK(11);
             __syncthreads();
-            FC_TICK(12);
             if (is_storer) {
                 // one box per lane; columns beyond the matrix edge (ragged tile) are clipped
                 // by the tensor map
@@ -666,7 +653,6 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
                 fk_bulk_commit();
             }
             store_pending = true;
-            FC_TICK(13);
         }
         if (ALIAS) {
             if (!TMA) __syncthreads();   // step 3 done with the shared buffer before the next tile lands in it
@@ -762,17 +748,18 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             if constexpr (DB) {
                 sStage = sStage0 + buf * STAGE_FLOATS;
                 bar = bar0 + 8u * (uint32_t)buf;
-                if (!fk_mbar_wait(bar, (phase >> buf) & 1u)) return;
+                if (!fk_wait_or_report(bar, (phase >> buf) & 1u, p.wait_cycles, p.status)) {
+                    // never landed: before the CTA's shared memory is released, wait (bounded)
+                    // for the load in flight into the other buffer as well
+                    if (tile + (int)gridDim.x < p.num_tiles)
+                        (void)fk_mbar_wait(bar0 + 8u * (uint32_t)(buf ^ 1), (phase >> (buf ^ 1)) & 1u, FK_WAIT_CYCLES);
+                    return;
+                }
                 phase ^= (1u << buf);
             } else {
-            if (!fk_mbar_wait(bar, phase)) return;
-            phase ^= 1u;
+                if (!fk_wait_or_report(bar, phase, p.wait_cycles, p.status)) return;
+                phase ^= 1u;
             }
-#ifdef FC_EXP_TMAONLY
-            __syncthreads();
-            if (is_fetcher && tile + (int)gridDim.x < p.num_tiles) fetch_tile(row_n, tcol_n);
-            continue;
-#endif
             // Rows ky = 0 and ky = N/2 are real after the column pass, so they travel through
             // the row pass as one complex row Z = X_0 + i X_{N/2}.  For N <= 32 the whole CTA
             // forms Z in the staging tile first (one element per thread, one more barrier), so
@@ -947,15 +934,18 @@ template <> struct FftCfg<32>  { static constexpr int G = 8;  static constexpr b
 template <> struct FftCfg<64>  { static constexpr int G = 4;  static constexpr bool ALIAS = false, SALIAS = false; static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = true; };
 template <> struct FftCfg<128> { static constexpr int G = 2;  static constexpr bool ALIAS = true,  SALIAS = false; static constexpr int MINB = 1, MINB_INV = 1; static constexpr bool TMA = false; };
 
+// SM count of the current device (0 on failure); looked up once per device ordinal.
 static inline int fft_sm_count() {
-    static int sms = 0;
-    if (sms == 0) {
-        int dev = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-            sms = 0;
+    static std::atomic<int> sms[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 0;
+    const bool slot = dev >= 0 && dev < 64;
+    int v = slot ? sms[dev].load(std::memory_order_relaxed) : 0;
+    if (v == 0) {
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        if (slot) sms[dev].store(v, std::memory_order_relaxed);
     }
-    return sms;
+    return v;
 }
 
 // Grid of a persistent kernel: one CTA per resident slot.  The attribute call and the

@@ -68,6 +68,7 @@ struct conv_plan_s {
     bool timed;             // a timed pass has been issued
     cudaEvent_t ev[5];
     bool ev_made;
+    long long wait_cycles;  // limit of a bounded device-side wait in SM cycles; 0 = the kernels' default
 };
 
 namespace {
@@ -223,8 +224,9 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         const bool fresh_a = (pass != PASS_ACCGRAD), fresh_b = (pass == PASS_FPROP);
         need_a = fresh_a || plan->cached[d.a.kind] != a_in;
         need_b = fresh_b || plan->cached[d.b.kind] != b_in;
-        plan->cached[d.a.kind] = a_in;
-        plan->cached[d.b.kind] = b_in;
+        // a spectrum counts as cached only once its transform has been launched (below)
+        if (need_a) plan->cached[d.a.kind] = nullptr;
+        if (need_b) plan->cached[d.b.kind] = nullptr;
     }
 
     auto operand = [&](const OperandDesc& o, const float* in, float* spec) {
@@ -234,6 +236,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         fp.R = o.spec.R; fp.C = o.spec.C; fp.ld = o.spec.ld;
         fp.win = o.win; fp.H = o.H; fp.W = o.W; fp.nty = o.nty; fp.ntx = o.ntx;
         fp.step_y = o.step_y; fp.step_x = o.step_x; fp.oy = o.oy; fp.ox = o.ox;
+        fp.status = status; fp.wait_cycles = plan->wait_cycles;
         return fp;
     };
     const bool timing = plan->timing && plan->ev_made;
@@ -269,12 +272,17 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         if (forward(fb, nullptr) != cudaSuccess) return FFTCONV_ECUDA;
     }
     mark(2);
+    if (plan->reuse) {
+        plan->cached[d.a.kind] = a_in;
+        plan->cached[d.b.kind] = b_in;
+    }
 
     fc::GemmParams gp{};
     gp.A = specA; gp.B = specB; gp.C = specC;
     gp.bins = plan->bins; gp.M = d.M; gp.N = d.N; gp.K = d.K;
     gp.lda = d.a.spec.ld; gp.ldb = d.b.spec.ld; gp.ldc = d.c.spec.ld;
     gp.transA = d.transA; gp.transB = d.transB; gp.conjA = d.conjA; gp.conjB = d.conjB;
+    gp.wait_cycles = plan->wait_cycles;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     // the kernels of a pass overlap their ramp-up with the predecessor's drain where that
     // was measured to pay (see dep_launch.cuh)
@@ -296,6 +304,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     ip.scale = 1.0f / ((float)plan->n * (float)plan->n);
     ip.accumulate = accumulate ? 1 : 0;
     ip.overlap = overlap ? 1 : 0;
+    ip.status = status; ip.wait_cycles = plan->wait_cycles;
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if ((big ? fc::launch_c2r_two_pass(plan->n, ip, scratch, scratch_bytes, st)
              : fc::launch_c2r<true>(plan->n, ip, st)) != cudaSuccess)
@@ -337,6 +346,7 @@ FFTCONV_API int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, in
     p->ws = nullptr; p->ws_bytes = 0;
     p->timing = 0; p->timed = false; p->ev_made = false;
     p->reuse = 0; p->cached[0] = p->cached[1] = p->cached[2] = nullptr;
+    p->wait_cycles = 0;
     if (frame_only) {
         // pick the tile basis now: the estimate ranks 8..64 against each other (the untiled
         // candidate does not exist), smallest admissible basis as the fallback
@@ -501,18 +511,21 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[FFTCONV_NOALLOC
 
 namespace {
 constexpr int kMaxDevices = 64;
-void* g_noalloc_ptr[kMaxDevices] = {nullptr};
+// Written at most once per device with one and the same value (the array's address on that
+// device), so concurrent first calls from several host threads agree; atomic so that the
+// race is a defined one.
+std::atomic<void*> g_noalloc_ptr[kMaxDevices];
 
 // Device address of the scratch array on the current device (nullptr on failure).
 void* noalloc_scratch_address() {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
-    if (!g_noalloc_ptr[dev]) {
-        void* ptr = nullptr;
+    void* ptr = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess) return nullptr;
-        g_noalloc_ptr[dev] = ptr;
+        g_noalloc_ptr[dev].store(ptr, std::memory_order_release);
     }
-    return g_noalloc_ptr[dev];
+    return ptr;
 }
 }  // namespace
 
@@ -562,6 +575,12 @@ FFTCONV_API int conv_plan_status(conv_plan_t* plan) {
         cudaMemset(plan->ws, 0, sizeof(int));
         return FFTCONV_EDEVICE_TIMEOUT;
     }
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_plan_set_wait_limit(conv_plan_t* plan, long long sm_cycles) {
+    if (!plan || sm_cycles < 0) return FFTCONV_EINVAL;
+    plan->wait_cycles = sm_cycles;
     return FFTCONV_OK;
 }
 
@@ -704,17 +723,3 @@ FFTCONV_API const char* fftconv_status_string(int status) {
 FFTCONV_API unsigned long long fftconv_launch_count(void) {
     return g_launches.load(std::memory_order_relaxed);
 }
-
-#ifdef FC_EXP_TIMELINE
-// Measurement builds only: cycle counts per phase of a forward tile loop (CTA 0, thread 0),
-// accumulated since the last reset.
-FFTCONV_API int fftconv_debug_timeline(long long* out16, int reset) {
-    if (out16 && cudaMemcpyFromSymbol(out16, fc::fc_timeline, sizeof(long long) * 16) != cudaSuccess)
-        return FFTCONV_ECUDA;
-    if (reset) {
-        long long zero[16] = {0};
-        if (cudaMemcpyToSymbol(fc::fc_timeline, zero, sizeof(zero)) != cudaSuccess) return FFTCONV_ECUDA;
-    }
-    return FFTCONV_OK;
-}
-#endif

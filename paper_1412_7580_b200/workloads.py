@@ -163,3 +163,55 @@ def shard_range(S: int, rank: int, world: int):
     base, extra = divmod(int(S), int(world))
     lo = rank * base + min(rank, extra)
     return lo, lo + base + (1 if rank < extra else 0)
+
+
+def plane_coords(dims, seed: int) -> np.ndarray:
+    """Three coordinates from every plane of a 4-D tensor [a, b, rows, cols]: one uniform
+    random element, one in the last row and one in the last column (the edges that a
+    mis-clipped tile would get wrong); int32 [3 * a * b, 4]."""
+    a, b, rows, cols = (int(d) for d in dims)
+    rng = np.random.default_rng([SEED_ROOT, 78, seed])
+    pa, pb = np.meshgrid(np.arange(a), np.arange(b), indexing="ij")
+    pa, pb = pa.ravel(), pb.ravel()
+    n = pa.size
+    parts = []
+    for r, c in ((rng.integers(0, rows, n), rng.integers(0, cols, n)),
+                 (np.full(n, rows - 1), rng.integers(0, cols, n)),
+                 (rng.integers(0, rows, n), np.full(n, cols - 1))):
+        parts.append(np.stack([pa, pb, r, c], axis=1))
+    return np.ascontiguousarray(np.concatenate(parts, axis=0), dtype=np.int32)
+
+
+def sweep_host_bytes(s: ConvShape) -> int:
+    """Bytes of the three input tensors and three results of a sweep point on the host."""
+    return 8 * (s.S * s.f * s.h * s.w + s.fp * s.f * s.kh * s.kw + s.S * s.fp * s.oh * s.ow)
+
+
+def sweep_stratified(per_n_large: int = 8, per_n_other: int = 6, count: int = 1000,
+                     max_host_bytes: int = 5 << 29):
+    """A stratified, seeded slice of the `count`-point sweep: for every basis n in
+    {16, 32, 64, 128}, `per_n_large` points whose S, f and f' are all >= 64 (many
+    contraction tiles) and `per_n_other` points from the rest (small shapes, where the plan
+    resolves to the FP32 contraction, included).  Points whose tensors exceed
+    `max_host_bytes` on the host are passed over, so that a time-boxed run is dominated by
+    the GPU and the oracle, not by drawing random numbers."""
+    pts = sweep_points(count)
+    order = np.random.default_rng([SEED_ROOT, 56]).permutation(len(pts))
+    out = []
+    for n in (16, 32, 64, 128):
+        large, other = [], []
+        for oi in order:
+            s = pts[int(oi)]
+            if s.n != n or sweep_host_bytes(s) > max_host_bytes:
+                continue
+            if min(s.S, s.f, s.fp) >= 64:
+                if len(large) < per_n_large:
+                    large.append(s)
+            elif len(other) < per_n_other:
+                other.append(s)
+        out.append(large + other)
+    # round robin over the bases, so that a run stopped early has still seen all of them
+    mixed = []
+    for i in range(max(len(g) for g in out)):
+        mixed.extend(g[i] for g in out if i < len(g))
+    return mixed

@@ -4,7 +4,8 @@ Tolerances (max |gpu - oracle| / max |oracle|): 1e-4 for the FP32 path, 5e-3
 for the TF32 tensor-core contraction.  Small shapes are compared element by
 element on full tensors; the benchmark-size layers are compared on a seeded
 sample of output coordinates (the oracle evaluates the plain definition at
-those coordinates) plus the adjoint identity on the full GPU tensors.
+those coordinates) plus the adjoint identity on the full GPU tensors; in the
+benchmark's own math mode they are also compared element by element.
 """
 import numpy as np
 import pytest
@@ -119,52 +120,93 @@ def test_accgrad_accumulates_two_pass_transforms():
     assert relerr(dw.cpu().numpy().astype(np.float64), ref) <= 1e-4
 
 
+def check_sampled(s, x, w, dy, y, dx, dw, eff, counts, seed):
+    """Sampled parity on full-size tensors: the oracle evaluates the plain definition at the
+    16 corners and uniform random coordinates of every result, and at three elements of EVERY
+    output plane (one random, one in the last row, one in the last column), so that a wrong
+    tile, plane group or clipped edge anywhere shows up."""
+    import oracle
+    from paper_1412_7580_b200 import workloads as wl
+    fns = (lambda c: oracle.fprop_at(x, w, c), lambda c: oracle.bprop_at(dy, w, s.h, s.w, c),
+           lambda c: oracle.accgrad_at(dy, x, s.kh, s.kw, c))
+    worst = []
+    for k, (got, fn) in enumerate(zip((y, dx, dw), fns)):
+        c = np.concatenate([wl.sample_coords(got.shape, counts[k], seed=seed + 10 * k),
+                            wl.plane_coords(got.shape, seed=seed + 10 * k + 1)], axis=0)
+        err = relerr(got[c[:, 0], c[:, 1], c[:, 2], c[:, 3]], fn(c))
+        assert err <= TOL[eff[k]], (s.name, ("fprop", "bprop", "accgrad")[k], err)
+        worst.append(err / TOL[eff[k]])
+    return max(worst)
+
+
 @pytest.mark.parametrize("cfg", [1, 2, 3])
-@pytest.mark.parametrize("math", [1, 2])
-def test_benchmark_layers_sampled(cfg, math):
-    """Full-size layers in the launch configuration the benchmark times."""
+def test_benchmark_layers_full_tensors(cfg):
+    """The three benchmark layers at full size, in the launch configuration and math mode the
+    benchmark times (AUTO = TF32 tensor cores), every element of y, dx and dw against the
+    float64 oracle."""
     import oracle
     from paper_1412_7580_b200 import workloads as wl
     s = wl.CONFIGS[cfg]
     x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
-    y, dx, dw, eff = run_gpu(s, x, w, dy, math)
-    tol = max(TOL[e] for e in eff)
+    y, dx, dw, eff = run_gpu(s, x, w, dy, 0)
+    assert eff == [2, 2, 2]
+    assert relerr(y, oracle.fprop(x, w)) <= TOL[eff[0]]
+    assert relerr(dx, oracle.bprop(dy, w, s.h, s.w)) <= TOL[eff[1]]
+    assert relerr(dw, oracle.accgrad(dy, x, s.kh, s.kw)) <= TOL[eff[2]]
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3])
+def test_benchmark_layers_fp32_sampled(cfg):
+    """The same layers with the FP32 contraction: sampled coordinates (corners, uniform,
+    three per output plane) plus the adjoint identity on the full GPU tensors."""
+    from paper_1412_7580_b200 import workloads as wl
+    s = wl.CONFIGS[cfg]
+    x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+    y, dx, dw, eff = run_gpu(s, x, w, dy, 1)
+    assert eff == [1, 1, 1]
     for got in (y, dx, dw):
         assert np.all(np.isfinite(got))
-    # normalisation: max-abs of the sampled oracle values (close to the tensor's)
-    cy = wl.sample_coords(y.shape, 4000, seed=cfg)
-    ry = oracle.fprop_at(x, w, cy)
-    assert relerr(y[cy[:, 0], cy[:, 1], cy[:, 2], cy[:, 3]], ry) <= TOL[eff[0]]
-    cx = wl.sample_coords(dx.shape, 4000, seed=cfg + 10)
-    rx = oracle.bprop_at(dy, w, s.h, s.w, cx)
-    assert relerr(dx[cx[:, 0], cx[:, 1], cx[:, 2], cx[:, 3]], rx) <= TOL[eff[1]]
-    cw = wl.sample_coords(dw.shape, 600, seed=cfg + 20)
-    rw = oracle.accgrad_at(dy, x, s.kh, s.kw, cw)
-    assert relerr(dw[cw[:, 0], cw[:, 1], cw[:, 2], cw[:, 3]], rw) <= TOL[eff[2]]
+    check_sampled(s, x, w, dy, y, dx, dw, eff, (4000, 4000, 600), seed=cfg)
     # adjoint identity on the full GPU tensors: <y,dy> = <x,dx> = <w,dw>
     a = float(np.sum(y * dy)); b = float(np.sum(dx * x)); c = float(np.sum(dw * w))
     scale = np.sqrt(float(np.sum(y * y)) * float(np.sum(dy.astype(np.float64) ** 2)))
-    assert abs(a - b) <= 10 * tol * scale and abs(a - c) <= 10 * tol * scale
+    assert abs(a - b) <= 10 * 1e-4 * scale and abs(a - c) <= 10 * 1e-4 * scale
 
 
-def test_sweep_subset():
-    """A seeded slice of the parameter sweep (small enough for the CPU oracle
-    on sampled coordinates), all three passes, default math mode."""
-    import oracle
+def test_sweep_stratified_slice():
+    """A stratified, seeded slice of the 1,000-point parameter sweep, all three passes, default
+    math mode: every basis n in {16, 32, 64, 128}, eight points per basis with S, f, f' >= 64
+    (many contraction tiles per bin) and six smaller ones (which include shapes the plan gives
+    to the FP32 contraction).  Time-boxed; the points come round robin over the bases."""
+    import time
     from paper_1412_7580_b200 import workloads as wl
-    pts = [s for s in wl.sweep_points(1000) if s.S * s.f * s.fp <= 16 * 64 * 64][:40]
-    assert len(pts) >= 20
+    pts = wl.sweep_stratified()
+    assert len(pts) >= 48
+    t0, done, maths, per_n = time.time(), 0, set(), {}
     for s in pts:
+        if time.time() - t0 > 240.0:
+            break
         x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
         y, dx, dw, eff = run_gpu(s, x, w, dy, 0)
-        cy = wl.sample_coords(y.shape, 300, seed=s.point)
-        assert relerr(y[cy[:, 0], cy[:, 1], cy[:, 2], cy[:, 3]], oracle.fprop_at(x, w, cy)) <= TOL[eff[0]], s
-        cx = wl.sample_coords(dx.shape, 300, seed=s.point + 1)
-        assert relerr(dx[cx[:, 0], cx[:, 1], cx[:, 2], cx[:, 3]],
-                      oracle.bprop_at(dy, w, s.h, s.w, cx)) <= TOL[eff[1]], s
-        cw = wl.sample_coords(dw.shape, 60, seed=s.point + 2)
-        assert relerr(dw[cw[:, 0], cw[:, 1], cw[:, 2], cw[:, 3]],
-                      oracle.accgrad_at(dy, x, s.kh, s.kw, cw)) <= TOL[eff[2]], s
+        for got in (y, dx, dw):
+            assert np.all(np.isfinite(got)), s
+        small = s.macs <= 2e9
+        if small:
+            import oracle
+            assert relerr(y, oracle.fprop(x, w)) <= TOL[eff[0]], s
+            assert relerr(dx, oracle.bprop(dy, w, s.h, s.w)) <= TOL[eff[1]], s
+            assert relerr(dw, oracle.accgrad(dy, x, s.kh, s.kw)) <= TOL[eff[2]], s
+        else:
+            check_sampled(s, x, w, dy, y, dx, dw, eff, (300, 300, 60), seed=s.point)
+        done += 1
+        maths.update(eff)
+        per_n[s.n] = per_n.get(s.n, 0) + 1
+        if min(s.S, s.f, s.fp) >= 64:
+            per_n[(s.n, "large")] = per_n.get((s.n, "large"), 0) + 1
+    assert done >= 40, (done, per_n)
+    assert maths == {1, 2}                      # both contraction kernels were exercised
+    for n in (16, 32, 64, 128):
+        assert per_n.get(n, 0) >= 8 and per_n.get((n, "large"), 0) >= 5, per_n
 
 
 @pytest.mark.parametrize("dims", [(6, 20, 24, 16, 16, 3, 3, 16), (4, 24, 40, 31, 31, 5, 5, 32),

@@ -5,9 +5,9 @@ memory where the convolution is needed (the framework's allocator owns the whole
 GPU, or an allocation -- which synchronises the device -- is not acceptable at
 that point).  For them the library carries a fixed 32 MiB scratch array of its
 own.  This test calls that entry point through the C ABI and checks it against
-the ordinary conv_fprop (caller-lent workspace) on two calls in a row with
-different inputs, so that nothing may depend on what the previous call left in
-the shared array.  It lives in the file pytest collects last: a failure here
+the ordinary conv_fprop (caller-lent workspace) and against the float64 oracle on
+two calls in a row with different inputs, so that nothing may depend on what the
+previous call left in the shared array.  It lives in the file pytest collects last: a failure here
 cannot hide any other test under `pytest -x`.
 """
 import numpy as np
@@ -42,8 +42,11 @@ def test_noalloc_matches_conv_fprop_on_two_calls_in_a_row():
     from paper_1412_7580_b200 import workloads as wl
     shapes = [wl.ConvShape("noalloc_a", 32, 16, 48, 13, 13, 3, 3, 16, cfg=8, point=1),   # tensor-core path
               wl.ConvShape("noalloc_b", 3, 5, 7, 27, 30, 5, 4, 32, cfg=8, point=2)]     # FP32 path, ragged
+    import oracle
     for s in shapes:
-        need = fc.conv_plan_workspace_bytes(fc.conv_plan(*s.args()))
+        sizing = fc.conv_plan(*s.args())
+        need = fc.conv_plan_workspace_bytes(sizing)
+        fc.conv_plan_destroy(sizing)
         assert need <= fc.binding.NOALLOC_BYTES
         for call in range(2):           # second call: other values, same shared scratch
             x, w = wl.make_x(s), wl.make_w(s)
@@ -53,6 +56,10 @@ def test_noalloc_matches_conv_fprop_on_two_calls_in_a_row():
             assert np.all(np.isfinite(got))
             err = np.max(np.abs(got - ref)) / np.max(np.abs(ref))
             assert err <= TOL[eff], (s.name, call, err)
+            # and against the plain definition: a defect shared by both entry points would
+            # pass the comparison above
+            want = oracle.fprop(x, w)
+            assert np.max(np.abs(got - want)) / np.max(np.abs(want)) <= TOL[eff], (s.name, call)
 
 
 def test_noalloc_refuses_plans_beyond_its_fixed_scratch():
