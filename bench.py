@@ -1,22 +1,34 @@
 #!/usr/bin/env python
 """Benchmark of the FFT-convolution hot path: one step = fprop + bprop + accGrad
-of one layer (all four kernels of each pass) on seeded synthetic tensors.
+of one layer (all kernels of each pass) on seeded synthetic tensors.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1] [--math auto]
-    python bench.py --impl reference ...     # the float64 CPU oracle on the host cores
+    python bench.py [--gpus N] [--steps K] [--warmup W]      # the whole contract, one JSON line
+    python bench.py --config 1 ...                           # one layer config only (0 tiny, 1 mid, 2 large-kernel, 3 deep)
+    python bench.py --shape S,f,fp,h,w,kh,kw,n [--tile t]    # a layer shape of your own
+    python bench.py --sweep-only --sweep-points 1000 --sweep-budget 900 --sweep-out gpurun_out/sweep.jsonl
+    python bench.py --fft2d | --fft1d                        # throughput of the bare transforms
+    python bench.py --impl reference ...                     # the float64 CPU oracle on the host cores
 
 Prints ONE JSON line.  `value` is the paper's throughput metric (equivalent
 time-domain multiply-adds per second, Section 4.2, times two flops) summed over
-the three passes, with the inputs resident in HBM; `e2e` is the same metric with
-the host<->device copies inside the timed region; `roofline` describes the
-kernel with the largest share of the step; `cpu_baseline` is the oracle timed
-on a bounded sample of the same workload.  Under torchrun every rank runs the
-same layer on its own minibatch (data parallel over S: fprop and bprop need no
-exchange, the weight gradient is summed with one NCCL all-reduce).
+the three passes, with the inputs resident in HBM, on the headline workload: the
+large-kernel layer, the largest of the single-GPU layer configs.  The timed
+region is `--steps` steps long and is repeated until at least a second of GPU
+time has been measured; `ms_per_step` is the median over those blocks.  `e2e` is
+the same metric with the host<->device copies inside the timed region;
+`roofline` describes the kernel with the largest share of the step;
+`cpu_baseline` is the oracle timed on a bounded sample of the same workload.
+Without `--config` / `--shape` the line also carries `configs` (the same
+measurements for all four layer configs) and `sweep` (a time-boxed, stratified
+run of the parameter sweep: per-pass roofline fractions per basis).  Under
+torchrun every rank runs the same layer on its own minibatch (data parallel over
+S: fprop and bprop need no exchange, the weight gradient is summed with one NCCL
+all-reduce).
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -30,39 +42,31 @@ if ROOT not in sys.path:
 
 METRIC = "conv_gflops_equivalent_3pass"
 UNIT = "GFLOP/s-equivalent"
+HEADLINE_CONFIG = 2                                         # the large-kernel layer
 FP32_FFMA_TFLOPS_NOMINAL = 148 * 128 * 2 * 1.965e9 / 1e12   # SMs x lanes x 2 flops x max clock
-# DRAM bytes (read + write) of one launch from the ncu captures summarised under profiles/,
-# keyed by (workload, kernel, pass); None where no capture exists.
-NCU_TRAFFIC = {
-    # (workload, kernel, pass): read + write, profiles/dram_traffic_per_launch_three_layer_configs.md
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "fprop"): 156.5e6,
-    ("mid_S128_f96_fp256_31x31_k5", "bin_contraction", "fprop"): 242.4e6,
-    ("mid_S128_f96_fp256_31x31_k5", "c2r_ifft", "fprop"): 193.9e6,
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "bprop"): 291.0e6,
-    ("mid_S128_f96_fp256_31x31_k5", "bin_contraction", "bprop"): 277.1e6,
-    ("mid_S128_f96_fp256_31x31_k5", "c2r_ifft", "bprop"): 54.4e6,
-    ("mid_S128_f96_fp256_31x31_k5", "r2c_fft_both_operands", "accgrad"): 286.9e6,
-    ("mid_S128_f96_fp256_31x31_k5", "bin_contraction", "accgrad"): 257.7e6,
-    ("mid_S128_f96_fp256_31x31_k5", "c2r_ifft", "accgrad"): 107.6e6,
-    ("largek_S128_f64_fp64_64x64_k11", "r2c_fft_both_operands", "fprop"): 293.1e6,
-    ("largek_S128_f64_fp64_64x64_k11", "bin_contraction", "fprop"): 290.4e6,
-    ("largek_S128_f64_fp64_64x64_k11", "c2r_ifft", "fprop"): 192.0e6,
-    ("largek_S128_f64_fp64_64x64_k11", "r2c_fft_both_operands", "bprop"): 251.9e6,
-    ("largek_S128_f64_fp64_64x64_k11", "bin_contraction", "bprop"): 290.1e6,
-    ("largek_S128_f64_fp64_64x64_k11", "c2r_ifft", "bprop"): 222.4e6,
-    ("largek_S128_f64_fp64_64x64_k11", "r2c_fft_both_operands", "accgrad"): 454.2e6,
-    ("largek_S128_f64_fp64_64x64_k11", "bin_contraction", "accgrad"): 324.1e6,
-    ("largek_S128_f64_fp64_64x64_k11", "c2r_ifft", "accgrad"): 69.3e6,
-    ("deep_S128_f384_fp384_13x13_k3", "r2c_fft_both_operands", "fprop"): 210.8e6,
-    ("deep_S128_f384_fp384_13x13_k3", "bin_contraction", "fprop"): 251.7e6,
-    ("deep_S128_f384_fp384_13x13_k3", "c2r_ifft", "fprop"): 56.8e6,
-    ("deep_S128_f384_fp384_13x13_k3", "r2c_fft_both_operands", "bprop"): 198.2e6,
-    ("deep_S128_f384_fp384_13x13_k3", "bin_contraction", "bprop"): 251.8e6,
-    ("deep_S128_f384_fp384_13x13_k3", "c2r_ifft", "bprop"): 57.1e6,
-    ("deep_S128_f384_fp384_13x13_k3", "r2c_fft_both_operands", "accgrad"): 114.6e6,
-    ("deep_S128_f384_fp384_13x13_k3", "bin_contraction", "accgrad"): 222.3e6,
-    ("deep_S128_f384_fp384_13x13_k3", "c2r_ifft", "accgrad"): 172.6e6,
+MIN_TIMED_MS = 1000.0                                       # GPU time measured per number
+MAX_BLOCKS = 400
+
+# DRAM bytes (read + write) of one launch from the ncu capture summarised in the profile named
+# below, keyed by (workload, kernel, pass).  The capture belongs to one state of the kernel
+# sources; `kernel_sources_sha256` is the digest of paper_1412_7580_b200/csrc at that state, and
+# the bench reports the figure only while the sources still have that digest.
+NCU_TRAFFIC_SOURCE = {
+    "profile": "profiles/dram_traffic_per_launch_three_layer_configs.md",
+    "kernel_sources_sha256": "unset",
 }
+NCU_TRAFFIC = {}
+
+
+def kernel_sources_digest():
+    """sha256 over the CUDA sources of the library, in name order."""
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_1412_7580_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        if name.endswith((".cu", ".cuh")):
+            with open(os.path.join(csrc, name), "rb") as fh:
+                h.update(name.encode() + b"\0" + fh.read())
+    return h.hexdigest()
 
 
 def load_peaks():
@@ -111,8 +115,19 @@ def pass_model(s, which, tile=0):
     }
 
 
+def config_dict(s, tile, world, workspace_bytes):
+    """The `config` object of the JSON line; both arms print the same one for the same workload."""
+    working_mb = (workspace_bytes + 8 * (s.S * s.f * s.h * s.w + s.fp * s.f * s.kh * s.kw +
+                                         s.S * s.fp * s.oh * s.ow)) / 1e6
+    return {"workload": s.name, "S": s.S, "f": s.f, "fprime": s.fp, "h": s.h, "w": s.w,
+            "kh": s.kh, "kw": s.kw, "n": s.n, "tile_basis": tile, "passes": "fprop+bprop+accgrad",
+            "parallelism": "dp%d over S" % world,
+            "l2": ("working set %.0f MB > 126 MB L2, no flush" % working_mb) if working_mb > 126
+                  else ("working set %.1f MB is L2-resident: the figure is launch latency" % working_mb)}
+
+
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi (query only) while a region runs."""
 
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
          "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
@@ -125,7 +140,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", self.uuid, "--query-gpu=" + self.Q,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -145,7 +160,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.12] or [l for (_, l) in self.lines]
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.05] or [l for (_, l) in self.lines]
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for l in rows:
@@ -187,11 +202,11 @@ def oracle_sample_run(s, x, w, dy, budget_s):
         nel = int(min(max(rate * budget_s / 3.0, 2048), 50_000_000))
         c = wl.sample_coords(dims[name], nel, seed=2)
         t = time.perf_counter(); fns[name](c); dt = time.perf_counter() - t
-        # bprop border elements have fewer valid taps; count the formula's nominal taps
+        # bprop border elements have fewer valid taps; the count is the formula's nominal taps
         total_macs += float(len(c)) * per[name]
         total_t += dt
         desc.append("%s:%d elems" % (name, len(c)))
-    return 2.0 * total_macs, total_t, ", ".join(desc)
+    return 2.0 * total_macs, total_t, ", ".join(desc) + " (nominal taps per element)"
 
 
 def run_reference(args, s):
@@ -212,13 +227,16 @@ def run_reference(args, s):
         vals.append(fl / t / 1e9); times.append(t)
     vals.sort()
     v = vals[len(vals) // 2]
+    import paper_1412_7580_b200 as fc
+    plan = fc.conv_plan(*s.args())              # host-only: sizes the workspace the GPU arm would use
+    cfg = config_dict(s, 0, args.gpus, fc.conv_plan_workspace_bytes(plan))
+    fc.conv_plan_destroy(plan)
     line = {
         "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": 1e3 * sum(times) / max(len(times), 1),
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic",
-        "config": {"workload": s.name, "sample": "per step: " + desc},
+        "data": "synthetic", "config": cfg,
         "cpu_baseline": {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": "per step: " + desc},
         "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -230,279 +248,473 @@ def run_reference(args, s):
 # ---------------------------------------------------------------------------
 # GPU arm
 # ---------------------------------------------------------------------------
-def run_ours(args, s):
-    import numpy as np
-    import torch
-    import paper_1412_7580_b200 as fc
-    from paper_1412_7580_b200 import workloads as wl
+class Bench:
+    def __init__(self, args):
+        import torch
+        self.torch = torch
+        self.args = args
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+        torch.cuda.set_device(self.local)
+        self.dist = None
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.init_process_group("nccl", device_id=torch.device("cuda", self.local))
+            self.dist = dist
+        self.peaks = load_peaks()
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        if self.dist is not None:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
 
-    peaks = load_peaks()
-    math = {"auto": fc.MATH_AUTO, "fp32": fc.MATH_FP32, "tf32": fc.MATH_TF32}[args.math]
-    x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
-    plan = fc.conv_plan(*s.args())
-    fc.conv_plan_set_math(plan, math)
-    if args.tile:
-        fc.conv_plan_set_tiling(plan, args.tile)      # -1: the plan chooses
-    tile = fc.conv_plan_tile_basis(plan)
-    ws = fc.conv_plan_alloc_workspace(plan)
-    eff = fc.conv_plan_effective_math(plan)
-    hx, hw_, hdy = (torch.from_numpy(a).pin_memory() for a in (x, w, dy))
-    xd, wd, dyd = hx.cuda(), hw_.cuda(), hdy.cuda()
-    y = torch.empty((s.S, s.fp, s.oh, s.ow), device="cuda")
-    dx = torch.empty((s.S, s.f, s.h, s.w), device="cuda")
-    dw = torch.empty((s.fp, s.f, s.kh, s.kw), device="cuda")
-    hy, hdx, hdw = (torch.empty(t.shape, dtype=torch.float32).pin_memory() for t in (y, dx, dw))
-
-    def step():
-        fc.conv_fprop(plan, xd, wd, y)
-        fc.conv_bprop(plan, dyd, wd, dx)
-        fc.conv_accgrad(plan, dyd, xd, dw)
-        if dist is not None:
-            dist.all_reduce(dw)        # data parallel over S: sum of the per-rank weight gradients
-
-    # End to end: every step copies x, w, dy from pinned host memory and y, dx, dw back.  The
-    # copies run on their own streams so that the two PCIe directions and the kernels overlap;
-    # each pass waits only for the tensors it reads, each read-back for the pass that wrote it.
-    main_stream = torch.cuda.current_stream()
-    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
-    ev = {k: torch.cuda.Event() for k in ("xw", "dy", "y", "dx", "dw")}
-
-    small = 4 * (x.size + w.size + dy.size) < (8 << 20)     # a few MB: stream hand-offs cost more than they hide
-
-    def step_e2e():
-        if small:
-            xd.copy_(hx, non_blocking=True); wd.copy_(hw_, non_blocking=True)
-            dyd.copy_(hdy, non_blocking=True)
-            step()
-            hy.copy_(y, non_blocking=True); hdx.copy_(dx, non_blocking=True)
-            hdw.copy_(dw, non_blocking=True)
-            return
-        s_in.wait_stream(main_stream)          # the previous step has read its inputs
-        with torch.cuda.stream(s_in):
-            xd.copy_(hx, non_blocking=True); wd.copy_(hw_, non_blocking=True)
-            ev["xw"].record(s_in)
-            dyd.copy_(hdy, non_blocking=True)
-            ev["dy"].record(s_in)
-        main_stream.wait_stream(s_out)         # the previous step's results have left the device
-        main_stream.wait_event(ev["xw"])
-        fc.conv_fprop(plan, xd, wd, y)
-        ev["y"].record(main_stream)
-        with torch.cuda.stream(s_out):
-            s_out.wait_event(ev["y"]); hy.copy_(y, non_blocking=True)
-        main_stream.wait_event(ev["dy"])
-        fc.conv_bprop(plan, dyd, wd, dx)
-        ev["dx"].record(main_stream)
-        with torch.cuda.stream(s_out):
-            s_out.wait_event(ev["dx"]); hdx.copy_(dx, non_blocking=True)
-        fc.conv_accgrad(plan, dyd, xd, dw)
-        if dist is not None:
-            dist.all_reduce(dw)
-        ev["dw"].record(main_stream)
-        with torch.cuda.stream(s_out):
-            s_out.wait_event(ev["dw"]); hdw.copy_(dw, non_blocking=True)
-
-    def e2e_drain():
-        main_stream.wait_stream(s_out)         # the timed region ends when the last result is on the host
-
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def timed(fn, steps, drain=None):
+    def timed_block(self, fn, steps, drain=None):
+        """One timed region of exactly `steps` calls: barrier + synchronize on both sides,
+        CUDA events on the launching stream, maximum over the ranks."""
+        torch = self.torch
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        barrier()
+        self.barrier()
         e0.record()
         for _ in range(steps):
             fn()
         if drain is not None:
             drain()
         e1.record()
-        barrier()
+        self.barrier()
         ms = e0.elapsed_time(e1)
-        if dist is not None:
+        if self.dist is not None:
             t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            self.dist.all_reduce(t, op=self.dist.ReduceOp.MAX)
             ms = float(t.item())
         return ms
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local).uuid).replace("GPU-", ""))
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.25)
-    launches0 = fc.fftconv_launch_count()
-    t0 = time.time()
-    ms_total = timed(step, args.steps)
-    # keep the GPU under the same load a little longer so the clock sampler sees it
-    reps = 0
-    while time.time() - t0 < 1.0 and reps < 200:
-        step(); reps += 1
-    torch.cuda.synchronize()
-    t1 = time.time()
-    # counted by the library.  Per pass: the forward FFTs (one launch for both operands with the
-    # one-pass kernels, one per operand with the two-pass kernels), the contraction, the inverse FFT
-    counted = fc.fftconv_launch_count() - launches0
-    assert counted % (args.steps + reps) == 0 and counted // (args.steps + reps) in (9, 12)
-    launches = counted // (args.steps + reps) * args.steps
-    clocks = sampler.stop(t0, t1) if rank == 0 else None
-    ms_step = ms_total / args.steps
+    def timed(self, fn, steps, drain=None, min_ms=MIN_TIMED_MS):
+        """Repeats the timed block until `min_ms` of GPU time has been measured (the number of
+        blocks is fixed from the first block, identical on every rank); returns the per-block
+        times in ms."""
+        first = self.timed_block(fn, steps, drain)
+        blocks = int(min(max(min_ms / max(first, 1e-3), 1), MAX_BLOCKS))
+        return [first] + [self.timed_block(fn, steps, drain) for _ in range(blocks - 1)]
 
-    for _ in range(2):
-        step_e2e()
-    ms_e2e = timed(step_e2e, args.steps, e2e_drain) / args.steps
-    assert fc.conv_plan_status(plan) == 0
+    # -- one layer config, all measurements ---------------------------------------------
+    def measure(self, s, math, tile_req=0, sample_clocks=False, reuse_line=True, cpu_budget=0.0):
+        import numpy as np
+        import paper_1412_7580_b200 as fc
+        from paper_1412_7580_b200 import workloads as wl
+        torch, args, world, dist = self.torch, self.args, self.world, self.dist
+        peaks = self.peaks
+        x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+        plan = fc.conv_plan(*s.args())
+        fc.conv_plan_set_math(plan, math)
+        if tile_req:
+            fc.conv_plan_set_tiling(plan, tile_req)      # -1: the plan chooses
+        tile = fc.conv_plan_tile_basis(plan)
+        ws = fc.conv_plan_alloc_workspace(plan)
+        eff = fc.conv_plan_effective_math(plan)
+        hx, hw_, hdy = (torch.from_numpy(a).pin_memory() for a in (x, w, dy))
+        xd, wd, dyd = hx.cuda(), hw_.cuda(), hdy.cuda()
+        y = torch.empty((s.S, s.fp, s.oh, s.ow), device="cuda")
+        dx = torch.empty((s.S, s.f, s.h, s.w), device="cuda")
+        dw = torch.empty((s.fp, s.f, s.kh, s.kw), device="cuda")
+        hy, hdx, hdw = (torch.empty(t.shape, dtype=torch.float32).pin_memory() for t in (y, dx, dw))
 
-    flops_step = 3 * 2.0 * s.macs
-    value = world * flops_step / (ms_step * 1e-3) / 1e9
-    e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e9
+        def step():
+            fc.conv_fprop(plan, xd, wd, y)
+            fc.conv_bprop(plan, dyd, wd, dx)
+            fc.conv_accgrad(plan, dyd, xd, dw)
+            if dist is not None:
+                dist.all_reduce(dw)        # data parallel over S: sum of the per-rank weight gradients
 
-    names = ["fprop", "bprop", "accgrad"]
-    calls = [lambda: fc.conv_fprop(plan, xd, wd, y), lambda: fc.conv_bprop(plan, dyd, wd, dx),
-             lambda: fc.conv_accgrad(plan, dyd, xd, dw)]
-    reps = max(args.steps, 10)
+        # End to end: every step copies x, w, dy from pinned host memory and y, dx, dw back.  The
+        # copies run on their own streams so that the two PCIe directions and the kernels overlap;
+        # each pass waits only for the tensors it reads, each read-back for the pass that wrote it.
+        main_stream = torch.cuda.current_stream()
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        ev = {k: torch.cuda.Event() for k in ("xw", "dy", "y", "dx", "dw")}
+        small = 4 * (x.size + w.size + dy.size) < (8 << 20)     # a few MB: stream hand-offs cost more than they hide
 
-    # per-pass durations, normal launch sequence, CUDA events on the launching stream
-    pass_ms = {n: [] for n in names}
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-           for _ in range(3 * reps)]
-    torch.cuda.synchronize()
-    k = 0
-    for _ in range(reps):
-        for c in calls:
-            evs[k][0].record(); c(); evs[k][1].record(); k += 1
-    torch.cuda.synchronize()
-    k = 0
-    for _ in range(reps):
-        for n in names:
-            pass_ms[n].append(evs[k][0].elapsed_time(evs[k][1])); k += 1
+        def step_e2e():
+            if small:
+                xd.copy_(hx, non_blocking=True); wd.copy_(hw_, non_blocking=True)
+                dyd.copy_(hdy, non_blocking=True)
+                step()
+                hy.copy_(y, non_blocking=True); hdx.copy_(dx, non_blocking=True)
+                hdw.copy_(dw, non_blocking=True)
+                return
+            s_in.wait_stream(main_stream)          # the previous step has read its inputs
+            with torch.cuda.stream(s_in):
+                xd.copy_(hx, non_blocking=True); wd.copy_(hw_, non_blocking=True)
+                ev["xw"].record(s_in)
+                dyd.copy_(hdy, non_blocking=True)
+                ev["dy"].record(s_in)
+            main_stream.wait_stream(s_out)         # the previous step's results have left the device
+            main_stream.wait_event(ev["xw"])
+            fc.conv_fprop(plan, xd, wd, y)
+            ev["y"].record(main_stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev["y"]); hy.copy_(y, non_blocking=True)
+            main_stream.wait_event(ev["dy"])
+            fc.conv_bprop(plan, dyd, wd, dx)
+            ev["dx"].record(main_stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev["dx"]); hdx.copy_(dx, non_blocking=True)
+            fc.conv_accgrad(plan, dyd, xd, dw)
+            if dist is not None:
+                dist.all_reduce(dw)
+            ev["dw"].record(main_stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev["dw"]); hdw.copy_(dw, non_blocking=True)
 
-    # per-kernel durations from CUDA events recorded by the library on its stream:
-    # mode 1 = the normal launch sequence (fused forward FFT, contraction, inverse FFT),
-    # mode 2 = the two forward FFTs launched apart (detail only)
-    def stage_times(mode):
-        fc.conv_plan_enable_stage_timing(plan, mode)
-        acc = {n: np.zeros(4) for n in names}
+        def e2e_drain():
+            main_stream.wait_stream(s_out)         # the timed region ends when the last result is on the host
+
+        warmup = max(args.warmup, 3)
+        for _ in range(warmup):
+            step()
+        sampler = None
+        if sample_clocks and self.rank == 0:
+            sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(self.local).uuid).replace("GPU-", ""))
+            sampler.start()
+            time.sleep(0.25)
+        launches0 = fc.fftconv_launch_count()
+        t0 = time.time()
+        blocks = self.timed(step, args.steps)
+        t1 = time.time()
+        # counted by the library.  Per pass: the forward FFTs (one launch for both operands with the
+        # one-pass kernels, one per operand with the two-pass kernels), the contraction, the inverse FFT
+        counted = fc.fftconv_launch_count() - launches0
+        total_steps = args.steps * len(blocks)
+        assert counted % total_steps == 0, (counted, total_steps)
+        launches = counted // len(blocks)
+        clocks = sampler.stop(t0, t1) if sampler is not None else None
+        ms_step = float(np.median(blocks)) / args.steps
+
+        for _ in range(2):
+            step_e2e()
+        e2e_blocks = self.timed(step_e2e, args.steps, e2e_drain, min_ms=MIN_TIMED_MS / 2)
+        ms_e2e = float(np.median(e2e_blocks)) / args.steps
+        assert fc.conv_plan_status(plan) == 0
+
+        flops_step = 3 * 2.0 * s.macs
+        value = world * flops_step / (ms_step * 1e-3) / 1e9
+        e2e_value = world * flops_step / (ms_e2e * 1e-3) / 1e9
+
+        names = ["fprop", "bprop", "accgrad"]
+        calls = [lambda: fc.conv_fprop(plan, xd, wd, y), lambda: fc.conv_bprop(plan, dyd, wd, dx),
+                 lambda: fc.conv_accgrad(plan, dyd, xd, dw)]
+        reps = max(args.steps, 20)
+
+        # per-pass durations, normal launch sequence, CUDA events on the launching stream
+        pass_ms = {n: [] for n in names}
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(3 * reps)]
+        torch.cuda.synchronize()
+        k = 0
         for _ in range(reps):
-            for n, c in zip(names, calls):
-                c()
-                acc[n] += np.array(fc.conv_plan_stage_times_ms(plan))
-        fc.conv_plan_enable_stage_timing(plan, 0)
-        return {n: acc[n] / reps for n in names}
-    st1, st2 = stage_times(1), stage_times(2)
+            for c in calls:
+                evs[k][0].record(); c(); evs[k][1].record(); k += 1
+        torch.cuda.synchronize()
+        k = 0
+        for _ in range(reps):
+            for n in names:
+                pass_ms[n].append(evs[k][0].elapsed_time(evs[k][1])); k += 1
 
-    tf32_peak = peaks["bf16_tflops_sustained"] / 2.0
-    p_tflops = tf32_peak if eff == fc.MATH_TF32 else FP32_FFMA_TFLOPS_NOMINAL
-    bw = peaks["hbm_gbs"] * 1e9
-    passes, best = {}, None
-    kernel_names = ["r2c_fft_both_operands", None, "bin_contraction", "c2r_ifft"]
-    for n in names:
-        m = pass_model(s, n, tile)
-        t_ms = float(np.median(pass_ms[n]))
-        t_roof = max(m["b_fft"] / bw, m["gemm_flops"] / (p_tflops * 1e12))
-        t_stage = max((m["b_fft"] + m["b_gemm"]) / bw, m["gemm_flops"] / (p_tflops * 1e12))
-        kbytes = [m["stage_bytes"][0] + m["stage_bytes"][1], 0, m["stage_bytes"][2], m["stage_bytes"][3]]
-        passes[n] = {
-            "ms": t_ms, "ms_min": float(np.min(pass_ms[n])),
-            "gflops_equiv": m["equiv_flops"] / (t_ms * 1e-3) / 1e9,
-            "roofline_us": t_roof * 1e6, "roofline_frac": t_roof / (t_ms * 1e-3),
-            "unfused_roofline_us": t_stage * 1e6, "unfused_roofline_frac": t_stage / (t_ms * 1e-3),
-            "kernel_ms": {kernel_names[k]: float(st1[n][k]) for k in (0, 2, 3)},
-            "forward_fft_apart_ms": {"A": float(st2[n][0]), "B": float(st2[n][1])},
-        }
-        for k in (0, 2, 3):
-            cand = (float(st1[n][k]), n, k, m, kbytes[k])
-            if best is None or cand[0] > best[0]:
-                best = cand
-    dur_ms, bn, bk, bm, bbytes = best
-    if bk == 2 and bm["gemm_flops"] / (p_tflops * 1e12) > bbytes / bw:
-        ach = bm["gemm_flops"] / (dur_ms * 1e-3) / 1e12
-        roof = {"bound": "tensor" if eff == fc.MATH_TF32 else "alu", "achieved": ach,
-                "peak": p_tflops, "unit": "TFLOP/s", "frac": ach / p_tflops}
-    else:
-        ach = bbytes / (dur_ms * 1e-3) / 1e9
-        roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": ach / peaks["hbm_gbs"]}
-    roof.update({"traffic": None if tile else NCU_TRAFFIC.get((s.name, kernel_names[bk], bn)),
-                 "kernel": "%s/%s" % (bn, kernel_names[bk]),
-                 "kernel_ms": dur_ms, "algorithmic_bytes": bbytes,
-                 "peak_source": peaks["source"] + (" sustained bf16 / 2" if roof["bound"] == "tensor" else "")})
+        # per-kernel durations from CUDA events recorded by the library on its stream:
+        # mode 1 = the normal launch sequence (fused forward FFT, contraction, inverse FFT),
+        # mode 2 = the two forward FFTs launched apart (detail only)
+        def stage_times(mode):
+            fc.conv_plan_enable_stage_timing(plan, mode)
+            acc = {n: np.zeros(4) for n in names}
+            for _ in range(reps):
+                for n, c in zip(names, calls):
+                    c()
+                    acc[n] += np.array(fc.conv_plan_stage_times_ms(plan))
+            fc.conv_plan_enable_stage_timing(plan, 0)
+            return {n: acc[n] / reps for n in names}
+        st1, st2 = stage_times(1), stage_times(2)
 
-    # extra (not the headline, which re-transforms every operand in every pass): the same
-    # step with the forward spectra shared between the passes of the step
-    reuse = None
-    if not args.no_reuse_line and not tile:
-        plan_r = fc.conv_plan(*s.args())
-        fc.conv_plan_set_math(plan_r, math)
-        fc.conv_plan_set_spectrum_reuse(plan_r, True)
-        ws_r = fc.conv_plan_alloc_workspace(plan_r)
+        tf32_peak = peaks["bf16_tflops_sustained"] / 2.0
+        p_tflops = tf32_peak if eff == fc.MATH_TF32 else FP32_FFMA_TFLOPS_NOMINAL
+        bw = peaks["hbm_gbs"] * 1e9
+        passes, best = {}, None
+        kernel_names = ["r2c_fft_both_operands", None, "bin_contraction", "c2r_ifft"]
+        for n in names:
+            m = pass_model(s, n, tile)
+            t_ms = float(np.median(pass_ms[n]))
+            t_roof = max(m["b_fft"] / bw, m["gemm_flops"] / (p_tflops * 1e12))
+            t_stage = max((m["b_fft"] + m["b_gemm"]) / bw, m["gemm_flops"] / (p_tflops * 1e12))
+            kbytes = [m["stage_bytes"][0] + m["stage_bytes"][1], 0, m["stage_bytes"][2], m["stage_bytes"][3]]
+            passes[n] = {
+                "ms": t_ms, "ms_min": float(np.min(pass_ms[n])),
+                "gflops_equiv": m["equiv_flops"] / (t_ms * 1e-3) / 1e9,
+                "roofline_us": t_roof * 1e6, "roofline_frac": t_roof / (t_ms * 1e-3),
+                "unfused_roofline_us": t_stage * 1e6, "unfused_roofline_frac": t_stage / (t_ms * 1e-3),
+                "kernel_ms": {kernel_names[k]: float(st1[n][k]) for k in (0, 2, 3)},
+                "forward_fft_apart_ms": {"A": float(st2[n][0]), "B": float(st2[n][1])},
+            }
+            for k in (0, 2, 3):
+                cand = (float(st1[n][k]), n, k, m, kbytes[k])
+                if best is None or cand[0] > best[0]:
+                    best = cand
+        dur_ms, bn, bk, bm, bbytes = best
+        if bk == 2 and bm["gemm_flops"] / (p_tflops * 1e12) > bbytes / bw:
+            ach = bm["gemm_flops"] / (dur_ms * 1e-3) / 1e12
+            roof = {"bound": "tensor" if eff == fc.MATH_TF32 else "alu", "achieved": ach,
+                    "peak": p_tflops, "unit": "TFLOP/s", "frac": ach / p_tflops}
+        else:
+            ach = bbytes / (dur_ms * 1e-3) / 1e9
+            roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach / peaks["hbm_gbs"]}
+        digest = kernel_sources_digest()
+        fresh = digest == NCU_TRAFFIC_SOURCE["kernel_sources_sha256"]
+        traffic = NCU_TRAFFIC.get("%s/%s/%s" % (s.name, kernel_names[bk], bn)) if (fresh and not tile) else None
+        roof.update({"traffic": traffic,
+                     "traffic_source": dict(NCU_TRAFFIC_SOURCE, current_kernel_sources_sha256=digest,
+                                            note=None if fresh else "kernel sources changed since the capture: no figure reported"),
+                     "kernel": "%s/%s" % (bn, kernel_names[bk]),
+                     "kernel_ms": dur_ms, "algorithmic_bytes": bbytes,
+                     "peak_source": peaks["source"] + (" sustained bf16 / 2" if roof["bound"] == "tensor" else "")})
 
-        def step_r():
-            fc.conv_fprop(plan_r, xd, wd, y)
-            fc.conv_bprop(plan_r, dyd, wd, dx)
-            fc.conv_accgrad(plan_r, dyd, xd, dw)
-        for _ in range(3):
-            step_r()
-        lr0 = fc.fftconv_launch_count()
-        ms_r = timed(step_r, args.steps) / args.steps
-        launches_r = (fc.fftconv_launch_count() - lr0) // args.steps
-        reuse = {"ms_per_step": ms_r, "value": world * flops_step / (ms_r * 1e-3) / 1e9, "unit": UNIT,
-                 "gpu_launches_per_step": launches_r, "workspace_bytes": int(ws_r.numel()),
-                 "note": "x, w, dy spectra computed once per step and shared by the three passes"}
-        fc.conv_plan_destroy(plan_r)
-        del ws_r
+        # extra (not the headline, which re-transforms every operand in every pass): the same
+        # step with the forward spectra shared between the passes of the step
+        reuse = None
+        if reuse_line and not tile:
+            plan_r = fc.conv_plan(*s.args())
+            fc.conv_plan_set_math(plan_r, math)
+            fc.conv_plan_set_spectrum_reuse(plan_r, True)
+            ws_r = fc.conv_plan_alloc_workspace(plan_r)
 
-    cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        import oracle
-        fl, t, desc = oracle_sample_run(s, x, w, dy, args.cpu_budget)
-        cpu = {"value": fl / t / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-               "sample": desc + " (sampled output elements of each pass, plain definition, float64)"}
+            def step_r():
+                fc.conv_fprop(plan_r, xd, wd, y)
+                fc.conv_bprop(plan_r, dyd, wd, dx)
+                fc.conv_accgrad(plan_r, dyd, xd, dw)
+            for _ in range(3):
+                step_r()
+            lr0 = fc.fftconv_launch_count()
+            ms_r = self.timed_block(step_r, args.steps) / args.steps
+            launches_r = (fc.fftconv_launch_count() - lr0) // args.steps
+            reuse = {"ms_per_step": ms_r, "value": world * flops_step / (ms_r * 1e-3) / 1e9, "unit": UNIT,
+                     "gpu_launches_per_step": launches_r, "workspace_bytes": int(ws_r.numel()),
+                     "note": "x, w, dy spectra computed once per step and shared by the three passes"}
+            fc.conv_plan_destroy(plan_r)
+            del ws_r
 
-    if rank == 0:
-        line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None,
-            "dtype": "tf32" if eff == fc.MATH_TF32 else "f32", "data": "synthetic",
-            "config": {"workload": s.name, "S": s.S, "f": s.f, "fprime": s.fp, "h": s.h, "w": s.w,
-                       "kh": s.kh, "kw": s.kw, "n": s.n, "tile_basis": tile,
-                       "passes": "fprop+bprop+accgrad",
-                       "parallelism": "dp%d over S" % world,
-                       "l2": "working set %.0f MB > 126 MB L2, no flush" % (
-                           (ws.numel() + 4 * (x.size + w.size + dy.size) * 2) / 1e6)},
+        cpu = None
+        if cpu_budget > 0 and self.rank == 0 and world == 1:
+            import oracle
+            fl, t, desc = oracle_sample_run(s, x, w, dy, cpu_budget)
+            cpu = {"value": fl / t / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                   "sample": desc + " (sampled output elements of each pass, plain definition, float64)"}
+
+        cfg = config_dict(s, tile, world, int(ws.numel()))
+        out = {
+            "value": value, "ms_per_step": ms_step, "blocks": len(blocks),
+            "ms_per_step_min_max": [min(blocks) / args.steps, max(blocks) / args.steps],
+            "dtype": "tf32" if eff == fc.MATH_TF32 else "f32", "config": cfg,
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e,
                     "h2d_bytes_per_step": int(4 * (x.size + w.size + dy.size)),
                     "d2h_bytes_per_step": int(4 * (y.numel() + dx.numel() + dw.numel()))},
             "gpu_launches": launches, "clocks": clocks, "roofline": roof, "cpu_baseline": cpu,
             "passes": passes, "step_with_spectrum_reuse": reuse,
         }
+        fc.conv_plan_destroy(plan)
+        del ws, xd, wd, dyd, y, dx, dw, hx, hw_, hdy, hy, hdx, hdw
+        torch.cuda.empty_cache()
+        return out
+
+    # -- workload 5: the parameter sweep, timing only ------------------------------------
+    def sweep(self, points, budget_s, out_path=None, tile="off", reps=5, max_gb=40.0):
+        """Per-pass times and roofline fractions of sweep points (no oracle here: parity of the
+        sweep is the job of the GPU tests; this run only checks that every result is finite).
+        `points` is a list of ConvShapes; stops when the time budget is used up."""
+        import numpy as np
+        import paper_1412_7580_b200 as fc
+        from paper_1412_7580_b200 import workloads as wl
+        torch = self.torch
+        bw = self.peaks["hbm_gbs"] * 1e9
+        t_start = time.time()
+        recs, skipped = [], 0
+        fh = open(out_path, "w") if out_path else None
+        for s in points:
+            if time.time() - t_start > budget_s:
+                break
+            B = s.n * (s.n // 2 + 1)
+            planes = s.S * s.f + s.fp * s.f + s.S * s.fp
+            real_b = 4 * (s.S * s.f * s.h * s.w + s.fp * s.f * s.kh * s.kw + s.S * s.fp * s.oh * s.ow)
+            if 8 * B * planes + 2 * real_b > max_gb * 1e9:
+                skipped += 1
+                continue
+            x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+            p = fc.conv_plan(*s.args())
+            if tile == "auto":
+                fc.conv_plan_set_tiling(p, fc.TILE_AUTO)
+            ws = fc.conv_plan_alloc_workspace(p)
+            xd, wd, dyd = (torch.from_numpy(a).cuda() for a in (x, w, dy))
+            y = torch.full((s.S, s.fp, s.oh, s.ow), float("nan"), device="cuda")
+            dx = torch.full((s.S, s.f, s.h, s.w), float("nan"), device="cuda")
+            dw = torch.full((s.fp, s.f, s.kh, s.kw), float("nan"), device="cuda")
+            calls = [lambda: fc.conv_fprop(p, xd, wd, y), lambda: fc.conv_bprop(p, dyd, wd, dx),
+                     lambda: fc.conv_accgrad(p, dyd, xd, dw)]
+            ms = []
+            for c in calls:
+                c()                                    # warm-up
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * reps)]
+                for r in range(reps):
+                    ev[2 * r].record(); c(); ev[2 * r + 1].record()
+                torch.cuda.synchronize()
+                ms.append(float(np.median([ev[2 * r].elapsed_time(ev[2 * r + 1]) for r in range(reps)])))
+            ok = fc.conv_plan_status(p) == 0 and all(bool(torch.isfinite(t).all().item()) for t in (y, dx, dw))
+            t_roof_ms = (real_b + 8 * B * planes) / bw * 1e3   # byte term of the roofline; flops never bind here
+            fr = [t_roof_ms / m for m in ms]
+            rec = {"point": s.point, "S": s.S, "f": s.f, "fp": s.fp, "h": s.h, "k": s.kh, "n": s.n,
+                   "tile_basis": fc.conv_plan_tile_basis(p),
+                   "math": ["tf32" if fc.conv_plan_pass_math(p, k) == fc.MATH_TF32 else "f32" for k in range(3)],
+                   "finite_and_status_ok": ok, "ms": ms, "roofline_frac": fr,
+                   "gflops_equiv": [2.0 * s.macs / (m * 1e-3) / 1e9 for m in ms]}
+            recs.append(rec)
+            if fh:
+                fh.write(json.dumps(rec) + "\n"); fh.flush()
+            fc.conv_plan_destroy(p)
+            del xd, wd, dyd, y, dx, dw, ws
+        if fh:
+            fh.close()
+        per_n = {}
+        for n in (16, 32, 64, 128):
+            for label, sel in (("all", lambda r: True),
+                               ("S_f_fp_ge_64", lambda r: min(r["S"], r["f"], r["fp"]) >= 64)):
+                v = np.array([min(r["roofline_frac"]) for r in recs if r["n"] == n and sel(r)])
+                if v.size:
+                    per_n["n%d_%s" % (n, label)] = {
+                        "points": int(v.size), "min": float(v.min()), "p10": float(np.percentile(v, 10)),
+                        "median": float(np.median(v))}
+        return {"points_done": len(recs), "points_requested": len(points),
+                "points_not_finite_or_status": sum(not r["finite_and_status_ok"] for r in recs),
+                "points_skipped_memory": skipped, "seconds": time.time() - t_start, "tile": tile,
+                "roofline_frac_min_over_passes": per_n,
+                "note": "roofline = FFT-stage bytes of the untiled method / measured HBM rate; parity of "
+                        "these points is checked by tests/test_gpu_conv.py::test_sweep_stratified_slice"}
+
+    # -- the bare transforms ----------------------------------------------------------------
+    def bare(self, which, mb):
+        """Throughput of fft2d_r2c / fft2d_c2r (n = 8..128) or fft1d_r2c / fft1d_c2r (n = 8..256)
+        on `mb` megabytes of samples per launch (larger than the L2)."""
+        import paper_1412_7580_b200 as fc
+        torch = self.torch
+        peak = self.peaks["hbm_gbs"]
+
+        def t_us(fn, reps=20):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps * 1e3
+        rows = []
+        sizes = (8, 16, 32, 64, 128) if which == "fft2d" else (8, 16, 32, 64, 128, 256)
+        for n in sizes:
+            if which == "fft2d":
+                batch = (mb << 20) // (n * n * 4)
+                x = torch.rand((batch, n, n), device="cuda")
+                X = torch.empty((batch, n, n // 2 + 1, 2), device="cuda")
+                y = torch.empty_like(x)
+                tf = t_us(lambda: fc.fft2d_r2c(x, X, n))
+                ti = t_us(lambda: fc.fft2d_c2r(X, y, n, 1.0 / (n * n)))
+            else:
+                batch = (mb << 20) // (n * 4)
+                x = torch.rand((batch, n), device="cuda")
+                X = torch.empty((batch, n // 2 + 1, 2), device="cuda")
+                y = torch.empty_like(x)
+                tf = t_us(lambda: fc.fft1d_r2c(x, X, n))
+                ti = t_us(lambda: fc.fft1d_c2r(X, y, n, 1.0 / n))
+            nbytes = (x.numel() + X.numel()) * 4
+            rows.append({"n": n, "batch": batch, "algorithmic_bytes": nbytes,
+                         "forward_us": tf, "forward_gbs": nbytes / tf / 1e3, "forward_frac": nbytes / tf / 1e3 / peak,
+                         "inverse_us": ti, "inverse_gbs": nbytes / ti / 1e3, "inverse_frac": nbytes / ti / 1e3 / peak})
+            del x, X, y
+        return {"transform": which, "mb_per_launch": mb, "peak_gbs": peak, "peak_source": self.peaks["source"],
+                "rows": rows}
+
+
+def run_ours(args):
+    import paper_1412_7580_b200 as fc
+    from paper_1412_7580_b200 import workloads as wl
+    b = Bench(args)
+    math = {"auto": fc.MATH_AUTO, "fp32": fc.MATH_FP32, "tf32": fc.MATH_TF32}[args.math]
+    single = args.config is not None or args.shape is not None
+    extras = not single and not args.no_extras and b.world == 1
+
+    if args.fft2d or args.fft1d:
+        print(json.dumps({"metric": "bare_transform_throughput", "unit": "GB/s", "n_gpus": 1,
+                          "data": "synthetic",
+                          "tables": [b.bare(w, args.mb) for w, on in (("fft2d", args.fft2d), ("fft1d", args.fft1d)) if on]}),
+              flush=True)
+        return
+    if args.sweep_only:
+        pts = wl.sweep_points(args.sweep_points)
+        import numpy as np
+        order = np.random.default_rng([wl.SEED_ROOT, 55]).permutation(len(pts))   # seeded order: a time-boxed run is an unbiased sample
+        res = b.sweep([pts[int(i)] for i in order], args.sweep_budget, args.sweep_out, args.sweep_tile)
+        print(json.dumps({"metric": "sweep_roofline_fraction", "n_gpus": 1, "data": "synthetic", "sweep": res}),
+              flush=True)
+        return
+
+    if args.shape:
+        dims = [int(v) for v in args.shape.split(",")]
+        assert len(dims) == 8, "--shape wants S,f,fp,h,w,kh,kw,n"
+        s = wl.ConvShape("custom_S%d_f%d_fp%d_%dx%d_k%dx%d_n%d" % tuple(dims), *dims, cfg=6,
+                         point=sum(dims), w_dist="fan_in", dy_dist="normal")
+    else:
+        s = wl.CONFIGS[HEADLINE_CONFIG if args.config is None else args.config]
+    head = b.measure(s, math, args.tile, sample_clocks=True, reuse_line=not args.no_reuse_line,
+                     cpu_budget=0.0 if args.no_cpu_baseline else args.cpu_budget)
+    line = {
+        "metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": b.world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": head["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": head["dtype"], "data": "synthetic",
+        "config": head["config"], "e2e": head["e2e"], "gpu_launches": head["gpu_launches"],
+        "clocks": head["clocks"], "roofline": head["roofline"], "cpu_baseline": head["cpu_baseline"],
+        "timed_blocks": head["blocks"], "ms_per_step_min_max": head["ms_per_step_min_max"],
+        "passes": head["passes"], "step_with_spectrum_reuse": head["step_with_spectrum_reuse"],
+    }
+    if extras:
+        cfgs = {}
+        for idx in (0, 1, 2, 3):
+            if idx == HEADLINE_CONFIG and not args.tile and math == fc.MATH_AUTO:
+                r = head
+            else:
+                r = b.measure(wl.CONFIGS[idx], fc.MATH_AUTO, 0, sample_clocks=True, reuse_line=False)
+            cfgs[wl.CONFIGS[idx].name] = {
+                "ms_per_step": r["ms_per_step"], "value": r["value"], "dtype": r["dtype"],
+                "gpu_launches": r["gpu_launches"], "clocks": r["clocks"], "timed_blocks": r["blocks"],
+                "e2e": r["e2e"], "roofline": r["roofline"],
+                "passes": {n: {k: p[k] for k in ("ms", "roofline_us", "roofline_frac", "unfused_roofline_frac",
+                                                 "gflops_equiv", "kernel_ms")}
+                           for n, p in r["passes"].items()}}
+        line["configs"] = cfgs
+        line["sweep"] = b.sweep(wl.sweep_stratified(), args.sweep_budget)
+    if b.rank == 0:
         print(json.dumps(line), flush=True)
-    if dist is not None:
-        dist.barrier()
-        dist.destroy_process_group()
+    if b.dist is not None:
+        b.dist.barrier()
+        b.dist.destroy_process_group()
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20, help="steps per timed block")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=1, help="0 tiny, 1 mid (default), 2 large-kernel, 3 deep")
+    ap.add_argument("--config", type=int, default=None,
+                    help="0 tiny, 1 mid, 2 large-kernel (the headline), 3 deep; given: that layer only")
     ap.add_argument("--shape", default=None,
                     help="S,f,fp,h,w,kh,kw,n : a layer shape of your own instead of --config "
                          "(seeded inputs as in the sweep; used for profiling single shapes)")
@@ -514,18 +726,22 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-reuse-line", action="store_true",
                     help="skip the extra measurement of a step with spectrum reuse between passes")
+    ap.add_argument("--no-extras", action="store_true", help="skip the `configs` and `sweep` keys")
+    ap.add_argument("--sweep-budget", type=float, default=75.0, help="seconds for the sweep")
+    ap.add_argument("--sweep-only", action="store_true", help="run the seeded sweep points only (timing)")
+    ap.add_argument("--sweep-points", type=int, default=1000)
+    ap.add_argument("--sweep-out", default=None, help="JSON lines, one per sweep point")
+    ap.add_argument("--sweep-tile", default="off", choices=["off", "auto"])
+    ap.add_argument("--fft2d", action="store_true", help="throughput table of the bare 2-D transforms")
+    ap.add_argument("--fft1d", action="store_true", help="throughput table of the bare 1-D transforms")
+    ap.add_argument("--mb", type=int, default=256, help="megabytes of samples per launch for --fft2d / --fft1d")
     args = ap.parse_args()
-    from paper_1412_7580_b200 import workloads as wl
-    s = wl.CONFIGS[args.config]
-    if args.shape:
-        dims = [int(v) for v in args.shape.split(",")]
-        assert len(dims) == 8, "--shape wants S,f,fp,h,w,kh,kw,n"
-        s = wl.ConvShape("custom_S%d_f%d_fp%d_%dx%d_k%dx%d_n%d" % tuple(dims), *dims, cfg=6,
-                         point=sum(dims), w_dist="fan_in", dy_dist="normal")
     if args.impl == "reference":
+        from paper_1412_7580_b200 import workloads as wl
+        s = wl.CONFIGS[HEADLINE_CONFIG if args.config is None else args.config]
         run_reference(args, s)
     else:
-        run_ours(args, s)
+        run_ours(args)
 
 
 if __name__ == "__main__":

@@ -8,6 +8,15 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def pytest_addoption(parser):
+    parser.addoption("--sweep-points", type=int, default=0,
+                     help="run tests/test_gpu_sweep_full.py on this many seeded sweep points (0: skip it)")
+    parser.addoption("--sweep-budget", type=float, default=1500.0, help="seconds for that run")
+    parser.addoption("--sweep-out", default=None, help="JSON lines of that run, one per point")
+    parser.addoption("--sweep-tile", default="off", choices=["off", "auto"],
+                     help="let every plan of that run choose a tile basis")
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200)")
 
