@@ -137,6 +137,15 @@ int conv_bprop(conv_plan_t* plan, const float* dy, const float* w, float* dx, vo
 int conv_accgrad(conv_plan_t* plan, const float* dy, const float* x, float* dw, int accumulate,
                  void* cuda_stream);
 
+/* Forward transform of small planes.  Operand planes of at most 13 x 13 samples (the filters
+ * of fprop and bprop) are transformed by a pruned separable DFT that evaluates one frequency
+ * bin for 32 adjacent planes at a time and writes whole 128-byte lines of the frequency-major
+ * spectrum (Section 5.1: the padding is never materialised -- here it is never even
+ * multiplied), instead of by the butterfly kernels that the large planes use.  On by default;
+ * enable == 0 sends every operand through the butterfly kernels (same results up to
+ * rounding).  The operand then has a launch of its own: a pass is four launches. */
+int conv_plan_set_small_plane_kernel(conv_plan_t* plan, int enable);
+
 /* Spectrum reuse across the passes of one training step (the paper's Section 6
  * notes that the forward transforms could be shared between passes, saving a
  * third of them, and passes on it for memory reasons).  With enable != 0 the

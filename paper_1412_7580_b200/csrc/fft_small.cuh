@@ -1,0 +1,241 @@
+// Forward 2-D R2C transform of SMALL planes (filters: kh x kw <= 13 x 13 samples padded
+// to n x n) straight into the frequency-major layout, as a pruned separable DFT.
+//
+// A filter plane has so few non-zero samples that its padded transform (Table 1, the
+// "FFT B" row; Section 5.1: the zero padding is never materialised) is cheaper as a direct
+// sum than as a butterfly network, and -- what matters on this machine -- the direct sum can
+// be organised around the STORES instead of around the planes: a warp takes 32 planes that
+// are adjacent along the minor index of the frequency-major matrix (lane = plane), every
+// lane evaluates the same frequency bin of its own plane at the same time, and the warp's
+// result for one (part, bin) is one contiguous 128-byte line, written from registers.  No
+// staging tile, no TMA box of short rows: every store is a whole line, which is the only
+// access size at which the memory system runs at its streaming rate.
+//
+// Per task (32 planes x a group of <= KY rows ky of the kept half ky <= n/2):
+//   1. the 32 planes (contiguous in the BDHW tensor) are copied to shared memory with
+//      coalesced loads; lane l then reads plane l at an odd pitch (no bank conflicts);
+//   2. column sums   T[ky][v] = sum_u w[u][v] e^{-2 pi i ky u / n}        (registers)
+//   3. row sums      X[ky][kx] = sum_v T[ky][v] e^{-2 pi i kx v / n}  for all kx, four
+//      outputs kx0 + m n/4 at a time: the samples are grouped by v mod 4 into four partial
+//      sums P_q (e^{-2 pi i (n/4) v / n} = (-i)^v), so that the four outputs cost one set of
+//      kw complex multiply-adds plus additions (one radix-4 decimation-in-frequency step).
+// Twiddles come from a 128-entry table in constant memory (evaluated in double at build
+// time); their index is lane-uniform, so they travel through the uniform datapath.
+// The kernel can be asked for a range of rows ky only, i.e. for a subset of the bins.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fft_core.cuh"
+#include "fft_kernels.cuh"
+
+namespace fc {
+
+constexpr int SMALL_MAX_K = 13;       // largest plane side this kernel takes
+// rows ky per task (upper bound): the column sums T[ky][v] of a task live in registers, so
+// wide planes get fewer rows; narrow ones more (the staging of the planes is then shared by more bins)
+constexpr int small_ky(int kw) { return kw <= 3 ? 6 : (kw <= 5 ? 4 : (kw <= 9 ? 3 : 2)); }
+constexpr int SMALL_WARPS = 4;        // warps per CTA, each with its own tasks
+
+struct TwTable128 { float2 v[128]; };
+constexpr TwTable128 make_tw128() {
+    TwTable128 t{};
+    for (int k = 0; k < 128; ++k) {
+        t.v[k].x = static_cast<float>(cx_cos2pi(k, 128));
+        t.v[k].y = static_cast<float>(cx_sin2pi(k, 128));
+    }
+    return t;
+}
+// (cos, sin) of 2 pi k / 128
+__constant__ TwTable128 c_tw128 = make_tw128();
+
+struct SmallParams {
+    const float* real_in;
+    float* spec_out;
+    int n, kh, kw;              // basis, plane rows, plane columns
+    int R, C, ld;               // frequency-major matrix: rows, cols (plane = row*C + col), leading dim
+    int ky_begin, ky_end;       // rows ky of the kept half [0, n/2] to produce
+    int groups;                 // tasks per block of 32 planes: the ky range in `groups` nearly equal parts
+    int cblocks;                // ceil(C / 32)
+    long long tasks;            // R * cblocks * groups
+    int pitch;                  // floats per plane in shared memory (odd)
+};
+
+template <int N, int KW>
+__global__ void __launch_bounds__(SMALL_WARPS * 32)
+r2c_small_kernel(const SmallParams p) {
+    extern __shared__ __align__(16) float sm_small[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* sw = sm_small + (size_t)warp * 32 * p.pitch;
+    constexpr int NC = N / 2 + 1, NQ = N / 4, TWS = 128 / N, MASK = N - 1, SMALL_KY = small_ky(KW);
+    const int ksq = p.kh * KW;
+    const size_t mat = (size_t)p.R * p.ld;              // floats per bin
+    const size_t part = (size_t)N * NC * mat;           // real parts -> imaginary parts
+    const int span = p.ky_end - p.ky_begin, base = span / p.groups, rem = span - base * p.groups;
+
+    dep_trigger();
+    dep_wait();                     // no global access above this line
+
+    const long long stride = (long long)gridDim.x * SMALL_WARPS;
+    for (long long t = (long long)blockIdx.x * SMALL_WARPS + warp; t < p.tasks; t += stride) {
+        const int g = (int)(t % p.groups);
+        const long long pb = t / p.groups;
+        const int cb = (int)(pb % p.cblocks), r = (int)(pb / p.cblocks);
+        const int c0 = cb * 32, count = min(32, p.C - c0);
+        const int ky0 = p.ky_begin + g * base + min(g, rem), kys = base + (g < rem ? 1 : 0);
+
+        // 1. stage the planes: `count` planes of ksq floats, contiguous in memory
+        __syncwarp();
+        {
+            const float* src = p.real_in + ((size_t)r * p.C + c0) * ksq;
+            const int total = count * ksq;
+            if (p.pitch == ksq) {
+                // odd plane size: the shared-memory image is the memory image
+                if ((reinterpret_cast<uintptr_t>(src) & 15) == 0) {
+                    const int vec = total >> 2;
+                    for (int e = lane; e < vec; e += 32)
+                        reinterpret_cast<float4*>(sw)[e] = __ldg(reinterpret_cast<const float4*>(src) + e);
+                    for (int e = 4 * vec + lane; e < total; e += 32) sw[e] = __ldg(src + e);
+                } else {
+                    for (int e = lane; e < total; e += 32) sw[e] = __ldg(src + e);
+                }
+            } else {
+                for (int pl = 0; pl < count; ++pl)
+                    for (int e = lane; e < ksq; e += 32) sw[pl * p.pitch + e] = __ldg(src + pl * ksq + e);
+            }
+        }
+        __syncwarp();
+        const float* mine = sw + (lane < count ? lane : 0) * p.pitch;
+
+        // 2. column sums for the rows ky0 .. ky0 + kys - 1 (absent rows computed and dropped)
+        float Tr[SMALL_KY][KW], Ti[SMALL_KY][KW];
+#pragma unroll
+        for (int j = 0; j < SMALL_KY; ++j)
+#pragma unroll
+            for (int v = 0; v < KW; ++v) Tr[j][v] = Ti[j][v] = 0.0f;
+        for (int u = 0; u < p.kh; ++u) {
+            float2 tw[SMALL_KY];
+#pragma unroll
+            for (int j = 0; j < SMALL_KY; ++j) tw[j] = c_tw128.v[(((ky0 + j) * u) & MASK) * TWS];
+#pragma unroll
+            for (int v = 0; v < KW; ++v) {
+                const float wv = mine[u * KW + v];
+#pragma unroll
+                for (int j = 0; j < SMALL_KY; ++j) {
+                    Tr[j][v] = fc_fma(wv, tw[j].x, Tr[j][v]);
+                    Ti[j][v] = fc_fma(-wv, tw[j].y, Ti[j][v]);
+                }
+            }
+        }
+
+        // 3. row sums, four outputs per step, one 128-byte line per (part, bin) and warp; the
+        //    twiddles are compile-time constants (immediate operands)
+        const bool live = lane < count;
+        // bin = kx * NC + ky; the four outputs of a step are NQ * NC bins apart
+        const size_t step = (size_t)NC * mat, quarter = (size_t)NQ * step;
+        float* o0 = p.spec_out + (size_t)ky0 * mat + (size_t)r * p.ld + c0 + lane;
+#pragma unroll
+        for (int j = 0; j < SMALL_KY; ++j) {
+            if (j >= kys) break;
+            float* o = o0 + (size_t)j * mat;
+            static_for<NQ>([&](auto KX0) {
+                constexpr int kx0 = decltype(KX0)::value;
+                float Pr[4] = {0.0f, 0.0f, 0.0f, 0.0f}, Pi[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                static_for<KW>([&](auto V) {
+                    constexpr int v = decltype(V)::value;
+                    // T[v] * e^{-i th}, th = 2 pi kx0 v / N:  (Tr c + Ti s, Ti c - Tr s)
+                    constexpr int idx = (kx0 * v) & MASK;
+                    constexpr float c = Tw<N, idx>::c, sn = Tw<N, idx>::s;
+                    if constexpr (idx == 0) {
+                        Pr[v & 3] += Tr[j][v]; Pi[v & 3] += Ti[j][v];
+                    } else {
+                        Pr[v & 3] = fc_fma(Tr[j][v], c, fc_fma(Ti[j][v], sn, Pr[v & 3]));
+                        Pi[v & 3] = fc_fma(Ti[j][v], c, fc_fma(-Tr[j][v], sn, Pi[v & 3]));
+                    }
+                });
+                // X[kx0 + m N/4] = sum_q (-i)^(q m) P_q
+                const float ar = Pr[0] + Pr[2], ai = Pi[0] + Pi[2], br = Pr[0] - Pr[2], bi = Pi[0] - Pi[2];
+                const float cr = Pr[1] + Pr[3], ci = Pi[1] + Pi[3], dr = Pr[1] - Pr[3], di = Pi[1] - Pi[3];
+                if (live) {
+                    float* q = o + (size_t)kx0 * step;
+                    q[0] = ar + cr;                 q[part] = ai + ci;                       // m = 0
+                    q[quarter] = br + di;           q[quarter + part] = bi - dr;             // m = 1: P0 - iP1 - P2 + iP3
+                    q[2 * quarter] = ar - cr;       q[2 * quarter + part] = ai - ci;         // m = 2
+                    q[3 * quarter] = br - di;       q[3 * quarter + part] = bi + dr;         // m = 3: P0 + iP1 - P2 - iP3
+                }
+            });
+        }
+    }
+}
+
+// True if the small-plane kernel takes this operand: planes that fill at most a quarter of
+// the basis (beyond that the butterfly kernels are as fast) and whose width has an instantiation.
+static inline bool small_supported(int n, int kh, int kw) {
+    if (n < 8 || n > 128 || kh < 1 || kw < 1 || kh > SMALL_MAX_K || kw > SMALL_MAX_K) return false;
+    if (2 * kh > n || 2 * kw > n) return false;
+    return kw <= 5 || kw == 7 || kw == 9 || kw == 11 || kw == 13;
+}
+
+template <int N, int KW>
+static cudaError_t launch_r2c_small_nk(const SmallParams& p, cudaStream_t st, bool overlap) {
+    if constexpr (2 * KW > N) {
+        return cudaErrorNotSupported;
+    } else {
+        auto kern = r2c_small_kernel<N, KW>;
+        const size_t smem = (size_t)SMALL_WARPS * 32 * p.pitch * sizeof(float);
+        int grid = 0;
+        const long long ctas = (p.tasks + SMALL_WARPS - 1) / SMALL_WARPS;
+        cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), SMALL_WARPS * 32, smem, ctas, &grid);
+        if (e != cudaSuccess) return e;
+        return dep_launch(overlap, kern, dim3(grid), dim3(SMALL_WARPS * 32), smem, st, p);
+    }
+}
+template <int N>
+static cudaError_t launch_r2c_small_n(const SmallParams& p, cudaStream_t st, bool overlap) {
+    switch (p.kw) {
+        case 1:  return launch_r2c_small_nk<N, 1>(p, st, overlap);
+        case 2:  return launch_r2c_small_nk<N, 2>(p, st, overlap);
+        case 3:  return launch_r2c_small_nk<N, 3>(p, st, overlap);
+        case 4:  return launch_r2c_small_nk<N, 4>(p, st, overlap);
+        case 5:  return launch_r2c_small_nk<N, 5>(p, st, overlap);
+        case 7:  return launch_r2c_small_nk<N, 7>(p, st, overlap);
+        case 9:  return launch_r2c_small_nk<N, 9>(p, st, overlap);
+        case 11: return launch_r2c_small_nk<N, 11>(p, st, overlap);
+        case 13: return launch_r2c_small_nk<N, 13>(p, st, overlap);
+    }
+    return cudaErrorNotSupported;
+}
+
+// Forward transform of one operand whose planes are small (see small_supported); produces the
+// rows ky in [ky_begin, ky_end) of the kept half, all kx.
+static cudaError_t launch_r2c_small(int n, const FftParams& f, int ky_begin, int ky_end, cudaStream_t st,
+                                    bool overlap = false) {
+    if (!small_supported(n, f.h, f.w) || f.win) return cudaErrorNotSupported;
+    if (ky_begin < 0 || ky_end > n / 2 + 1 || ky_begin >= ky_end) return cudaErrorInvalidValue;
+    SmallParams p{};
+    p.real_in = f.real_in; p.spec_out = f.spec_out;
+    p.n = n; p.kh = f.h; p.kw = f.w;
+    p.R = f.R; p.C = f.C; p.ld = f.ld;
+    p.ky_begin = ky_begin; p.ky_end = ky_end;
+    const int span = ky_end - ky_begin;
+    p.cblocks = (f.C + 31) / 32;
+    // rows ky per task: as many as SMALL_KY (the column sums are shared by them), fewer when
+    // the operand has too few planes to fill the machine with tasks otherwise
+    int ky_per = small_ky(f.w);
+    const long long blocks = (long long)f.R * p.cblocks, want = (long long)fft_sm_count() * 24;
+    while (ky_per > 1 && blocks * ((span + ky_per - 1) / ky_per) < want) --ky_per;
+    p.groups = (span + ky_per - 1) / ky_per;
+    p.tasks = blocks * p.groups;
+    p.pitch = (f.h * f.w) | 1;
+    switch (n) {
+        case 8:   return launch_r2c_small_n<8>(p, st, overlap);
+        case 16:  return launch_r2c_small_n<16>(p, st, overlap);
+        case 32:  return launch_r2c_small_n<32>(p, st, overlap);
+        case 64:  return launch_r2c_small_n<64>(p, st, overlap);
+        case 128: return launch_r2c_small_n<128>(p, st, overlap);
+    }
+    return cudaErrorNotSupported;
+}
+
+}  // namespace fc

@@ -15,6 +15,7 @@
 #include "cgemm_tc.cuh"
 #include "fft_kernels.cuh"
 #include "fft_big.cuh"
+#include "fft_small.cuh"
 #include "fft1d.cuh"
 
 #define FFTCONV_API extern "C" __attribute__((visibility("default")))
@@ -69,6 +70,7 @@ struct conv_plan_s {
     cudaEvent_t ev[5];
     bool ev_made;
     long long wait_cycles;  // limit of a bounded device-side wait in SM cycles; 0 = the kernels' default
+    int small_planes;       // small operand planes (filters) take the pruned-DFT forward kernel
 };
 
 namespace {
@@ -246,6 +248,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     const bool big = !tiled && fc::big_uses_two_pass(plan->n);
     float* scratch = reinterpret_cast<float*>(base + align_up(spectra_bytes(plan), kAlign));
     const size_t scratch_bytes = tiled ? 0 : fc::big_scratch_bytes(plan->n);
+    // One forward launch: both operands in one kernel (one-pass transforms), or one operand.
     auto forward = [&](const fc::FftParams& pa, const fc::FftParams* pb) -> cudaError_t {
         g_launches.fetch_add((big && pb) ? 2 : 1, std::memory_order_relaxed);
         if (!big) return fc::launch_r2c<true>(plan->n, pa, pb, st);
@@ -253,24 +256,34 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         if (e == cudaSuccess && pb) e = fc::launch_r2c_two_pass(plan->n, *pb, scratch, scratch_bytes, st);
         return e;
     };
+    // Small planes (the filters of fprop and bprop) take the pruned-DFT kernel, whose stores are
+    // whole 128-byte lines; it runs after the other operand's transform, as its programmatic
+    // dependent where that transform is a one-pass kernel.
+    auto is_small = [&](const fc::FftParams& f) {
+        return plan->small_planes && !f.win && fc::small_supported(plan->n, f.h, f.w);
+    };
+    auto forward_small = [&](const fc::FftParams& f, bool dep) -> cudaError_t {
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return fc::launch_r2c_small(plan->n, f, 0, plan->n / 2 + 1, st, dep && !big && !timing);
+    };
     mark(0);
     const fc::FftParams fa = operand(d.a, a_in, specA), fb = operand(d.b, b_in, specB);
-    if (!need_a || !need_b) {
-        // spectrum reuse: at most one operand left to transform
-        if (need_a || need_b) {
-            if (forward(need_a ? fa : fb, nullptr) != cudaSuccess) return FFTCONV_ECUDA;
-        }
-        mark(1);
-    } else if (!timing || plan->timing == 1) {
+    const bool small_a = need_a && is_small(fa), small_b = need_b && is_small(fb);
+    bool forward_last_small = false;
+    if (need_a && !small_a && need_b && !small_b && (!timing || plan->timing == 1)) {
         // both forward transforms in one launch: one ramp-up, one tail
         if (forward(fa, &fb) != cudaSuccess) return FFTCONV_ECUDA;
         mark(1);
     } else {
-        // timing mode 2: one kernel per operand, to time the two transforms apart
-        if (forward(fa, nullptr) != cudaSuccess) return FFTCONV_ECUDA;
+        // one kernel per operand (small planes, spectrum reuse, or timing mode 2)
+        bool launched = false;
+        if (need_a && !small_a) { if (forward(fa, nullptr) != cudaSuccess) return FFTCONV_ECUDA; launched = true; }
+        if (need_a && small_a) { if (forward_small(fa, launched) != cudaSuccess) return FFTCONV_ECUDA; launched = true; forward_last_small = true; }
         mark(1);
-        if (forward(fb, nullptr) != cudaSuccess) return FFTCONV_ECUDA;
+        if (need_b && !small_b) { if (forward(fb, nullptr) != cudaSuccess) return FFTCONV_ECUDA; launched = true; forward_last_small = false; }
+        if (need_b && small_b) { if (forward_small(fb, launched) != cudaSuccess) return FFTCONV_ECUDA; forward_last_small = true; }
     }
+    (void)forward_last_small;
     mark(2);
     if (plan->reuse) {
         plan->cached[d.a.kind] = a_in;
@@ -347,6 +360,7 @@ FFTCONV_API int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, in
     p->timing = 0; p->timed = false; p->ev_made = false;
     p->reuse = 0; p->cached[0] = p->cached[1] = p->cached[2] = nullptr;
     p->wait_cycles = 0;
+    p->small_planes = 1;
     if (frame_only) {
         // pick the tile basis now: the estimate ranks 8..64 against each other (the untiled
         // candidate does not exist), smallest admissible basis as the fallback
@@ -581,6 +595,12 @@ FFTCONV_API int conv_plan_status(conv_plan_t* plan) {
 FFTCONV_API int conv_plan_set_wait_limit(conv_plan_t* plan, long long sm_cycles) {
     if (!plan || sm_cycles < 0) return FFTCONV_EINVAL;
     plan->wait_cycles = sm_cycles;
+    return FFTCONV_OK;
+}
+
+FFTCONV_API int conv_plan_set_small_plane_kernel(conv_plan_t* plan, int enable) {
+    if (!plan) return FFTCONV_EINVAL;
+    plan->small_planes = enable ? 1 : 0;
     return FFTCONV_OK;
 }
 
