@@ -146,6 +146,14 @@ int conv_accgrad(conv_plan_t* plan, const float* dy, const float* x, float* dw, 
  * rounding).  The operand then has a launch of its own: a pass is four launches. */
 int conv_plan_set_small_plane_kernel(conv_plan_t* plan, int enable);
 
+/* Filter spectrum through the cache (Section 6 asks for fewer passes over memory between the
+ * stages).  With chunks > 1, fprop and bprop transform the filters and contract them in
+ * `chunks` ranges of frequency rows, one after the other: each part of the filter spectrum
+ * is consumed by the contraction right after it was produced, while it is still in the L2
+ * cache.  Needs the small-plane kernel and the tensor-core contraction; otherwise, and with
+ * chunks <= 1, the pass runs unchunked.  Results do not depend on the setting. */
+int conv_plan_set_filter_chunks(conv_plan_t* plan, int chunks);
+
 /* Spectrum reuse across the passes of one training step (the paper's Section 6
  * notes that the forward transforms could be shared between passes, saving a
  * third of them, and passes on it for memory reasons).  With enable != 0 the

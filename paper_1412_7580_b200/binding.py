@@ -23,7 +23,7 @@ EXPORTS = (
     "conv_plan_set_workspace", "conv_plan_set_spectrum_reuse", "conv_plan_invalidate_spectra",
     "conv_plan_set_tiling", "conv_plan_tile_basis",
     "conv_fprop", "conv_fprop_noalloc", "conv_bprop", "conv_accgrad", "conv_plan_status",
-    "conv_plan_set_wait_limit", "conv_plan_set_small_plane_kernel",
+    "conv_plan_set_wait_limit", "conv_plan_set_small_plane_kernel", "conv_plan_set_filter_chunks",
     "conv_plan_destroy", "conv_plan_enable_stage_timing", "conv_plan_stage_times_ms", "fft2d_r2c", "fft2d_c2r", "fft1d_r2c", "fft1d_c2r", "fftconv_bin_contract",
     "fftconv_status_string", "fftconv_launch_count",
 )
@@ -65,6 +65,7 @@ def lib():
         L.conv_plan_status.argtypes = [p]
         L.conv_plan_set_wait_limit.argtypes = [p, ctypes.c_longlong]
         L.conv_plan_set_small_plane_kernel.argtypes = [p, i]
+        L.conv_plan_set_filter_chunks.argtypes = [p, i]
         L.conv_plan_destroy.argtypes = [p]
         L.conv_plan_enable_stage_timing.argtypes = [p, i]
         L.conv_plan_stage_times_ms.argtypes = [p, p]
@@ -251,8 +252,13 @@ def conv_plan_status(plan: Plan) -> int:
 
 def conv_plan_set_small_plane_kernel(plan: Plan, enable=True) -> None:
     """Pruned-DFT forward kernel for operand planes of at most 13 x 13 samples (default on)."""
-    _check(lib().conv_plan_set_small_plane_kernel(plan.handle, int(bool(enable))),
+    _check(lib().conv_plan_set_small_plane_kernel(plan.handle, int(enable)),
            "conv_plan_set_small_plane_kernel")
+
+
+def conv_plan_set_filter_chunks(plan: Plan, chunks: int) -> None:
+    """fprop / bprop: transform and contract the filters in this many ranges of frequency rows."""
+    _check(lib().conv_plan_set_filter_chunks(plan.handle, int(chunks)), "conv_plan_set_filter_chunks")
 
 
 def conv_plan_set_wait_limit(plan: Plan, sm_cycles: int) -> None:

@@ -28,6 +28,10 @@ struct GemmParams {
     int conjA, conjB;     // use the complex conjugate of the operand
     int overlap;          // host only: launch as a programmatic dependent of the previous kernel
     long long wait_cycles; // host only: limit of a bounded wait in the tensor-core kernel (<= 0: default)
+    // Tensor-core kernel only: contract a subset of the bins.  Bins are numbered kx * nc + ky;
+    // with ky_count > 0 only the rows ky in [ky_begin, ky_begin + ky_count) of every kx are
+    // contracted (bins / nc values of kx).  ky_count == 0: all bins.
+    int nc, ky_begin, ky_count;
 };
 
 constexpr int FG_BM = 64, FG_BN = 64, FG_BK = 16, FG_PAD = 4, FG_T = 256;

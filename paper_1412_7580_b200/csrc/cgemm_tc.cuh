@@ -59,6 +59,8 @@ struct TcParams {
     int conjA, conjB;
     int* status;
     long long wait_cycles;      // limit of one wait in SM clock cycles (the draining waits keep TC_WAIT_CYCLES)
+    int bins_run;               // bins contracted by this launch (all of them, or a ky range of every kx)
+    int nc, ky_begin, ky_count; // ky_count > 0: local bin b -> kx = b / ky_count, ky = ky_begin + b % ky_count
 };
 
 static inline bool tc_shape_supported(int M, int N, int K) {
@@ -227,7 +229,13 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const uint32_t tmem_base = *tmem_slot;
     dep_wait();                     // no global access above this line
 
-    const int num_tiles = p.bins * p.m_tiles * p.n_tiles;
+    const int num_tiles = p.bins_run * p.m_tiles * p.n_tiles;
+    // local bin of this launch -> bin of the spectra
+    auto global_bin = [&](int b) {
+        if (p.ky_count == 0) return b;
+        const int kx = b / p.ky_count;
+        return kx * p.nc + p.ky_begin + (b - kx * p.ky_count);
+    };
     auto give_up = [&]() {
         *abort_flag = 1;
         if (p.status) atomicExch(p.status, 1);
@@ -241,7 +249,7 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             for (int t = blockIdx.x; ok && t < num_tiles; t += gridDim.x) {
                 const int n_t = t % p.n_tiles;
                 const int m_t = (t / p.n_tiles) % p.m_tiles;
-                const int bin = t / (p.n_tiles * p.m_tiles);
+                const int bin = global_bin(t / (p.n_tiles * p.m_tiles));
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
                     const int s = it % TC_STAGES;
                     const uint32_t ph = (uint32_t)(it / TC_STAGES) & 1u;
@@ -344,7 +352,7 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         for (int t = blockIdx.x; ok && t < num_tiles; t += gridDim.x, ++tl) {
             const int n_t = t % p.n_tiles;
             const int m_t = (t / p.n_tiles) % p.m_tiles;
-            const int bin = t / (p.n_tiles * p.m_tiles);
+            const int bin = global_bin(t / (p.n_tiles * p.m_tiles));
             const int buf = tl & 1;
             if (!mbar_wait(tfull(buf), (uint32_t)(tl >> 1) & 1u, abort_flag, p.wait_cycles)) { ok = false; break; }
             tc_fence_after_sync();
@@ -431,7 +439,13 @@ static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStrea
     p.conjA = g.conjA; p.conjB = g.conjB;
     p.status = status;
     p.wait_cycles = g.wait_cycles > 0 ? g.wait_cycles : TC_WAIT_CYCLES;
-    const long long tiles = (long long)p.bins * p.m_tiles * p.n_tiles;
+    p.bins_run = g.bins; p.nc = g.nc; p.ky_begin = g.ky_begin; p.ky_count = 0;
+    if (g.ky_count > 0) {
+        if (g.nc < 1 || g.bins % g.nc != 0 || g.ky_begin < 0 || g.ky_begin + g.ky_count > g.nc)
+            return cudaErrorInvalidValue;
+        if (g.ky_count < g.nc) { p.ky_count = g.ky_count; p.bins_run = (g.bins / g.nc) * g.ky_count; }
+    }
+    const long long tiles = (long long)p.bins_run * p.m_tiles * p.n_tiles;
     if (tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
     return dep_launch(g.overlap != 0, kern, dim3(grid), dim3(TC_THREADS), TC_SMEM_BYTES, st, tmA, tmB, tmC, p);

@@ -60,6 +60,7 @@ struct SmallParams {
     int cblocks;                // ceil(C / 32)
     long long tasks;            // R * cblocks * groups
     int pitch;                  // floats per plane in shared memory (odd)
+    int concurrent;             // launched to run beside its predecessor: do not wait for it (see launch_r2c_small)
 };
 
 template <int N, int KW>
@@ -75,7 +76,10 @@ r2c_small_kernel(const SmallParams p) {
     const int span = p.ky_end - p.ky_begin, base = span / p.groups, rem = span - base * p.groups;
 
     dep_trigger();
-    dep_wait();                     // no global access above this line
+    // `concurrent`: the predecessor in the stream is the other operand's forward transform, which
+    // this kernel neither reads from nor overwrites; the launch that follows both is a plain one
+    // and therefore waits for both.
+    if (!p.concurrent) dep_wait();  // no global access above this line
 
     const long long stride = (long long)gridDim.x * SMALL_WARPS;
     for (long long t = (long long)blockIdx.x * SMALL_WARPS + warp; t < p.tasks; t += stride) {
@@ -209,8 +213,11 @@ static cudaError_t launch_r2c_small_n(const SmallParams& p, cudaStream_t st, boo
 
 // Forward transform of one operand whose planes are small (see small_supported); produces the
 // rows ky in [ky_begin, ky_end) of the kept half, all kx.
+// overlap: launch as a programmatic dependent of the previous kernel.  concurrent (with overlap):
+// additionally skip the wait for that kernel, so that the two run side by side; the caller must
+// then launch the next kernel the plain way (a plain launch waits for everything before it).
 static cudaError_t launch_r2c_small(int n, const FftParams& f, int ky_begin, int ky_end, cudaStream_t st,
-                                    bool overlap = false) {
+                                    bool overlap = false, bool concurrent = false) {
     if (!small_supported(n, f.h, f.w) || f.win) return cudaErrorNotSupported;
     if (ky_begin < 0 || ky_end > n / 2 + 1 || ky_begin >= ky_end) return cudaErrorInvalidValue;
     SmallParams p{};
@@ -228,6 +235,7 @@ static cudaError_t launch_r2c_small(int n, const FftParams& f, int ky_begin, int
     p.groups = (span + ky_per - 1) / ky_per;
     p.tasks = blocks * p.groups;
     p.pitch = (f.h * f.w) | 1;
+    p.concurrent = (overlap && concurrent) ? 1 : 0;
     switch (n) {
         case 8:   return launch_r2c_small_n<8>(p, st, overlap);
         case 16:  return launch_r2c_small_n<16>(p, st, overlap);

@@ -16,6 +16,7 @@
 #include "fft_kernels.cuh"
 #include "fft_big.cuh"
 #include "fft_small.cuh"
+#include "fft_sub.cuh"
 #include "fft1d.cuh"
 
 #define FFTCONV_API extern "C" __attribute__((visibility("default")))
@@ -71,6 +72,7 @@ struct conv_plan_s {
     bool ev_made;
     long long wait_cycles;  // limit of a bounded device-side wait in SM cycles; 0 = the kernels' default
     int small_planes;       // small operand planes (filters) take the pruned-DFT forward kernel
+    int filter_chunks;      // > 1: the filter spectrum is produced and contracted in this many bin ranges
 };
 
 namespace {
@@ -251,7 +253,11 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     // One forward launch: both operands in one kernel (one-pass transforms), or one operand.
     auto forward = [&](const fc::FftParams& pa, const fc::FftParams* pb) -> cudaError_t {
         g_launches.fetch_add((big && pb) ? 2 : 1, std::memory_order_relaxed);
-        if (!big) return fc::launch_r2c<true>(plan->n, pa, pb, st);
+        if (!big) {
+            // wide planes at n = 64: the sub-batched kernels (rows twice as long); else the plain ones
+            const cudaError_t es = fc::launch_r2c_sub_any(plan->n, pa, pb, st);
+            return es != cudaErrorNotSupported ? es : fc::launch_r2c<true>(plan->n, pa, pb, st);
+        }
         cudaError_t e = fc::launch_r2c_two_pass(plan->n, pa, scratch, scratch_bytes, st);
         if (e == cudaSuccess && pb) e = fc::launch_r2c_two_pass(plan->n, *pb, scratch, scratch_bytes, st);
         return e;
@@ -262,14 +268,59 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     auto is_small = [&](const fc::FftParams& f) {
         return plan->small_planes && !f.win && fc::small_supported(plan->n, f.h, f.w);
     };
+    // dep: another forward transform of this pass was launched just before; the small-plane kernel
+    // then runs beside it (neither touches the other's data) and the contraction is launched the
+    // plain way, which waits for both.
+    bool forward_concurrent = false;
     auto forward_small = [&](const fc::FftParams& f, bool dep) -> cudaError_t {
         g_launches.fetch_add(1, std::memory_order_relaxed);
-        return fc::launch_r2c_small(plan->n, f, 0, plan->n / 2 + 1, st, dep && !big && !timing);
+        const bool conc = dep && !big && !timing && plan->small_planes == 1;
+        if (conc) forward_concurrent = true;
+        return fc::launch_r2c_small(plan->n, f, 0, plan->n / 2 + 1, st, conc, conc);
     };
     mark(0);
     const fc::FftParams fa = operand(d.a, a_in, specA), fb = operand(d.b, b_in, specB);
     const bool small_a = need_a && is_small(fa), small_b = need_b && is_small(fb);
-    bool forward_last_small = false;
+    const bool tensor = resolve_math(*plan, d) == FFTCONV_MATH_TF32;
+    // the kernels of a pass overlap their ramp-up with the predecessor's drain where that
+    // was measured to pay (see dep_launch.cuh)
+    const bool overlap = !big && !timing && (tensor || plan->n >= 32 || d.K <= 64);
+
+    fc::GemmParams gp{};
+    gp.A = specA; gp.B = specB; gp.C = specC;
+    gp.bins = plan->bins; gp.M = d.M; gp.N = d.N; gp.K = d.K;
+    gp.lda = d.a.spec.ld; gp.ldb = d.b.spec.ld; gp.ldc = d.c.spec.ld;
+    gp.transA = d.transA; gp.transB = d.transB; gp.conjA = d.conjA; gp.conjB = d.conjB;
+    gp.wait_cycles = plan->wait_cycles;
+    gp.nc = plan->n / 2 + 1;
+
+    const int nc = plan->n / 2 + 1;
+    const int chunks = (plan->filter_chunks > 1 && small_b && tensor && !timing)
+                           ? (plan->filter_chunks < nc ? plan->filter_chunks : nc) : 1;
+    if (chunks > 1) {
+        // Filter spectrum through the L2: the small-plane kernel can produce any range of rows
+        // ky, so the filter operand is transformed and contracted range by range -- each part
+        // of its spectrum is read back by the contraction right after it was written, while it
+        // is still in the cache, instead of crossing HBM twice.
+        bool launched = false;
+        if (need_a) {
+            if ((small_a ? forward_small(fa, false) : forward(fa, nullptr)) != cudaSuccess) return FFTCONV_ECUDA;
+            launched = true;
+        }
+        for (int c = 0; c < chunks; ++c) {
+            const int ky0 = (int)((long long)nc * c / chunks), ky1 = (int)((long long)nc * (c + 1) / chunks);
+            g_launches.fetch_add(2, std::memory_order_relaxed);
+            if (fc::launch_r2c_small(plan->n, fb, ky0, ky1, st, launched && !big) != cudaSuccess) return FFTCONV_ECUDA;
+            launched = true;
+            gp.ky_begin = ky0; gp.ky_count = ky1 - ky0;
+            gp.overlap = big ? 0 : 1;
+            if (fc::launch_cgemm_tc(gp, status, st) != cudaSuccess) return FFTCONV_ECUDA;
+        }
+        if (plan->reuse) {
+            plan->cached[d.a.kind] = a_in;
+            plan->cached[d.b.kind] = b_in;
+        }
+    } else {
     if (need_a && !small_a && need_b && !small_b && (!timing || plan->timing == 1)) {
         // both forward transforms in one launch: one ramp-up, one tail
         if (forward(fa, &fb) != cudaSuccess) return FFTCONV_ECUDA;
@@ -278,34 +329,24 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         // one kernel per operand (small planes, spectrum reuse, or timing mode 2)
         bool launched = false;
         if (need_a && !small_a) { if (forward(fa, nullptr) != cudaSuccess) return FFTCONV_ECUDA; launched = true; }
-        if (need_a && small_a) { if (forward_small(fa, launched) != cudaSuccess) return FFTCONV_ECUDA; launched = true; forward_last_small = true; }
+        if (need_a && small_a) { if (forward_small(fa, launched) != cudaSuccess) return FFTCONV_ECUDA; launched = true; }
         mark(1);
-        if (need_b && !small_b) { if (forward(fb, nullptr) != cudaSuccess) return FFTCONV_ECUDA; launched = true; forward_last_small = false; }
-        if (need_b && small_b) { if (forward_small(fb, launched) != cudaSuccess) return FFTCONV_ECUDA; forward_last_small = true; }
+        if (need_b && !small_b) { if (forward(fb, nullptr) != cudaSuccess) return FFTCONV_ECUDA; launched = true; }
+        if (need_b && small_b) { if (forward_small(fb, launched) != cudaSuccess) return FFTCONV_ECUDA; }
     }
-    (void)forward_last_small;
     mark(2);
     if (plan->reuse) {
         plan->cached[d.a.kind] = a_in;
         plan->cached[d.b.kind] = b_in;
     }
-
-    fc::GemmParams gp{};
-    gp.A = specA; gp.B = specB; gp.C = specC;
-    gp.bins = plan->bins; gp.M = d.M; gp.N = d.N; gp.K = d.K;
-    gp.lda = d.a.spec.ld; gp.ldb = d.b.spec.ld; gp.ldc = d.c.spec.ld;
-    gp.transA = d.transA; gp.transB = d.transB; gp.conjA = d.conjA; gp.conjB = d.conjB;
-    gp.wait_cycles = plan->wait_cycles;
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    // the kernels of a pass overlap their ramp-up with the predecessor's drain where that
-    // was measured to pay (see dep_launch.cuh)
-    const bool tensor = resolve_math(*plan, d) == FFTCONV_MATH_TF32;
-    const bool overlap = !big && !timing && (tensor || plan->n >= 32 || d.K <= 64);
-    gp.overlap = (overlap && (need_a || need_b)) ? 1 : 0;       // predecessor: this pass's forward transforms
+    // predecessor: this pass's forward transforms (plain launch after two that ran side by side)
+    gp.overlap = (overlap && (need_a || need_b) && !forward_concurrent) ? 1 : 0;
     cudaError_t ge;
     if (tensor) ge = fc::launch_cgemm_tc(gp, status, st);
     else ge = fc::launch_cgemm_ffma(gp, st);
     if (ge != cudaSuccess) return FFTCONV_ECUDA;
+    }
     mark(3);
 
     fc::FftParams ip{};
@@ -361,6 +402,7 @@ FFTCONV_API int conv_plan(conv_plan_t** out, int S, int f, int fprime, int h, in
     p->reuse = 0; p->cached[0] = p->cached[1] = p->cached[2] = nullptr;
     p->wait_cycles = 0;
     p->small_planes = 1;
+    p->filter_chunks = 1;
     if (frame_only) {
         // pick the tile basis now: the estimate ranks 8..64 against each other (the untiled
         // candidate does not exist), smallest admissible basis as the fallback
@@ -598,9 +640,15 @@ FFTCONV_API int conv_plan_set_wait_limit(conv_plan_t* plan, long long sm_cycles)
     return FFTCONV_OK;
 }
 
+FFTCONV_API int conv_plan_set_filter_chunks(conv_plan_t* plan, int chunks) {
+    if (!plan || chunks < 0) return FFTCONV_EINVAL;
+    plan->filter_chunks = chunks < 1 ? 1 : chunks;
+    return FFTCONV_OK;
+}
+
 FFTCONV_API int conv_plan_set_small_plane_kernel(conv_plan_t* plan, int enable) {
     if (!plan) return FFTCONV_EINVAL;
-    plan->small_planes = enable ? 1 : 0;
+    plan->small_planes = enable < 0 ? 0 : (enable > 2 ? 1 : enable);   // 2: without running beside the other transform (measurements)
     return FFTCONV_OK;
 }
 

@@ -73,8 +73,8 @@ def test_reuse_matches_plain_passes_and_oracle(dims):
     fc.conv_plan_invalidate_spectra(p)
     before = fc.fftconv_launch_count()
     fc.conv_accgrad(p, dyd, x3d, dw1)
-    # both operands afresh: one fused launch for large planes, one launch each for small ones
-    assert fc.fftconv_launch_count() - before == (4 if max(s.h, s.w) <= 13 else 3)
+    # both operands afresh, in one fused launch
+    assert fc.fftconv_launch_count() - before == 3
     torch.cuda.synchronize()
     assert relerr(dw1.cpu().numpy().astype(np.float64), oracle.accgrad(dy2, x3, s.kh, s.kw)) <= TOL[eff[2]]
     fc.conv_plan_destroy(p)
