@@ -252,7 +252,7 @@ def conv_plan_status(plan: Plan) -> int:
 
 def conv_plan_set_small_plane_kernel(plan: Plan, enable=True) -> None:
     """Pruned-DFT forward kernel for operand planes of at most 13 x 13 samples (default on)."""
-    _check(lib().conv_plan_set_small_plane_kernel(plan.handle, int(enable)),
+    _check(lib().conv_plan_set_small_plane_kernel(plan.handle, int(bool(enable))),
            "conv_plan_set_small_plane_kernel")
 
 

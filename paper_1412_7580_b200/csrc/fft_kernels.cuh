@@ -53,8 +53,22 @@
 namespace fc {
 
 // LAYOUT_FREQ_TMA / _DIRECT: planar frequency-major spectra, moved by the TMA or
-// by plain per-thread accesses; LAYOUT_BARE: [plane][n][n/2+1] interleaved pairs.
-enum { LAYOUT_FREQ_TMA = 0, LAYOUT_BARE = 1, LAYOUT_FREQ_DIRECT = 2 };
+// by plain per-thread accesses; LAYOUT_BARE: [plane][n][n/2+1] interleaved pairs, accessed
+// by the threads directly; LAYOUT_BARE_STAGED: the same layout, but a tile's planes (which
+// are contiguous in memory) travel between global and shared memory as one bulk
+// asynchronous copy per plane and the threads only touch the shared-memory image.
+enum { LAYOUT_FREQ_TMA = 0, LAYOUT_BARE = 1, LAYOUT_FREQ_DIRECT = 2, LAYOUT_BARE_STAGED = 3 };
+
+// Pitch (in complex elements) of one plane of the bare layout in shared memory: the plane
+// itself, rounded up so that every plane starts on a 16-byte boundary, plus a few elements so
+// that lanes running over the planes of a tile and over adjacent rows hit distinct banks.
+template <int N, int G>
+struct BareGeom {
+    static constexpr int PLANE = N * (N / 2 + 1);
+    static constexpr int SKEW = (G >= 8) ? 2 : 16 / G;
+    static constexpr int P2 = ((PLANE + 15) / 16) * 16 + SKEW;
+    static constexpr size_t BYTES = (((size_t)G * P2 * 8 + 127) / 128) * 128;
+};
 
 struct FftParams {
     const float* real_in;   // forward: real planes in
@@ -167,6 +181,10 @@ __device__ __forceinline__ void fk_bulk_g2s(uint32_t dst, const void* src, uint3
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
         ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
+__device__ __forceinline__ void fk_bulk_s2g(void* dst, uint32_t src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void fk_tma_load_3d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
                                                int c2, uint32_t bar) {
     asm volatile(
@@ -256,6 +274,9 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
     constexpr int T = N * G, NC = N / 2 + 1, M = N / 2, HALF = T / 2, B = N * NC;
     constexpr int PW = MidGeom<N, G>::PW, P = MidGeom<N, G>::P;
     constexpr bool TMA = (LAYOUT == LAYOUT_FREQ_TMA);
+    constexpr bool BSTG = (LAYOUT == LAYOUT_BARE_STAGED);
+    constexpr bool BARE = (LAYOUT == LAYOUT_BARE) || BSTG;
+    constexpr int P2 = BareGeom<N, G>::P2;
     constexpr int D = tma_bins_per_box(N);
     // The packed row (ky = 0 with ky = N/2) is taken apart either by the two threads that
     // transformed it or, with the TMA staging, afterwards by the whole CTA (one more barrier,
@@ -420,7 +441,8 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
         if (pending) {
             if (!fk_wait_or_report(bar, phase, p0.wait_cycles, p0.status)) {
                 // the copy never landed: let the stores already issued finish and leave
-                if (TMA && store_pending && is_storer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+                if ((TMA || BSTG) && store_pending && (TMA ? is_storer : tid >= T - 32))
+                    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
                 return;
             }
             phase ^= 1u;
@@ -501,7 +523,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
                     cfft<L, false>(br, bi);             // br/bi[k] = X[ky = 4k + q4]
                 }
             }
-            if (TMA && store_pending && is_storer) fk_bulk_wait_read();  // staging tile free again
+            if ((TMA || BSTG) && store_pending && (TMA ? is_storer : tid >= T - 32)) fk_bulk_wait_read();  // staging tile free again
             __syncthreads();   // tile consumed (and the previous tile's step 3 is done with sMid)
             if (!ALIAS) pending = (next < total_tiles) ? stage(second_n, row_n, tcol_n) : false;
             // Rows ky = 0 and ky = N/2 of a real column transform are real: they share the
@@ -553,7 +575,7 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             if constexpr (TMA && SALIAS) __syncthreads();   // scratch consumed: it becomes the staging tile
             cfft<M, false>(ar, ai);                     // ar/ai[k] = F[kx = 2k+q]
 
-            if constexpr (LAYOUT != LAYOUT_BARE) {
+            if constexpr (!BARE) {
                 // element (part, bin = kx*NC + ky, plane g): staging offset (part*B + bin)*G + g,
                 // global offset ((part*B + bin)*R + row)*ld + col
                 float* o;
@@ -595,8 +617,9 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
                 }
             } else {
                 // conventional half [ky][kx <= N/2]; the other rows come from the mirror bin
-                float2* base = reinterpret_cast<float2*>(p.spec_out) +
-                               ((size_t)row * p.C + c0 + gB) * (size_t)(N * NC);
+                float2* base = BSTG ? reinterpret_cast<float2*>(sStage) + gB * P2
+                                    : reinterpret_cast<float2*>(p.spec_out) +
+                                          ((size_t)row * p.C + c0 + gB) * (size_t)(N * NC);
                 if (!packed) {
                     static_for<M>([&](auto Kk) {
                         constexpr int k = decltype(Kk)::value;
@@ -654,13 +677,27 @@ r2c_kernel(const __grid_constant__ CUtensorMap tmS0, const __grid_constant__ CUt
             }
             store_pending = true;
         }
+        if constexpr (BSTG) {
+            // the planes of the tile are contiguous in memory: one bulk copy per plane, issued
+            // by the lanes of the last warp
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncthreads();
+            if (tid >= T - 32 && (tid & 31) < gcount) {
+                const int g = tid & 31;
+                fk_bulk_s2g(reinterpret_cast<float2*>(p.spec_out) + ((size_t)row * p.C + c0 + g) * (size_t)(N * NC),
+                            fk_smem_u32(reinterpret_cast<float2*>(sStage) + g * P2), (uint32_t)(N * NC * 8));
+                fk_bulk_commit();
+            }
+            store_pending = true;
+        }
         if (ALIAS) {
             if (!TMA) __syncthreads();   // step 3 done with the shared buffer before the next tile lands in it
             pending = (next < total_tiles) ? stage(second_n, row_n, tcol_n) : false;
             __syncthreads();
         }
     }
-    if (TMA && store_pending && is_storer) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    if ((TMA || BSTG) && store_pending && (TMA ? is_storer : tid >= T - 32))
+        asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
 }
 
 // ---------------------------------------------------------------------------
@@ -675,6 +712,8 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
     constexpr int T = N * G, NC = N / 2 + 1, M = N / 2, HALF = T / 2, B = N * NC;
     constexpr int PW = MidGeom<N, G>::PW, P = MidGeom<N, G>::P;
     constexpr bool TMA = (LAYOUT == LAYOUT_FREQ_TMA);
+    constexpr bool BSTG = (LAYOUT == LAYOUT_BARE_STAGED);
+    constexpr int P2 = BareGeom<N, G>::P2;
     constexpr int D = tma_bins_per_box(N);
     static_assert(!DB || TMA, "double-buffered staging needs the TMA layout");
     constexpr int STAGE_FLOATS = 2 * B * G;
@@ -712,10 +751,22 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
         }
     };
     auto fetch_tile = [&](int row, int tcol) { fetch_into(row, tcol, sStage, bar); };
+    // bare layout, staged: the planes of a tile are contiguous in memory; one bulk copy per plane
+    auto fetch_bare = [&](int row, int tcol) {                                   // whole last warp
+        const int c0 = tcol * G, cnt = min(G, p.C - c0);
+        if ((tid & 31) == 0) fk_mbar_expect_tx(bar0, (uint32_t)(cnt * N * NC * 8));
+        __syncwarp();
+        if ((tid & 31) < cnt) {
+            const int g = tid & 31;
+            fk_bulk_g2s(fk_smem_u32(reinterpret_cast<float2*>(sStage0) + g * P2),
+                        reinterpret_cast<const float2*>(p.spec_in) + ((size_t)row * p.C + c0 + g) * (size_t)(N * NC),
+                        (uint32_t)(N * NC * 8), bar0);
+        }
+    };
     uint32_t phase = 0;             // DB: bit b is the phase of buffer b's barrier
     int row = blockIdx.x / tpr, tcol = blockIdx.x - (blockIdx.x / tpr) * tpr;
     dep_trigger();
-    if constexpr (TMA) {
+    if constexpr (TMA || BSTG) {
         if (tid == 0) {
             fk_mbar_init(bar0, 1);
             if (DB) fk_mbar_init(bar0 + 8u, 1);
@@ -723,7 +774,11 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
         }
         __syncthreads();
         dep_wait();                 // no global access above this line
-        if (is_fetcher && blockIdx.x < p.num_tiles) fetch_tile(row, tcol);
+        if constexpr (BSTG) {
+            if (is_fetcher && blockIdx.x < p.num_tiles) fetch_bare(row, tcol);
+        } else {
+            if (is_fetcher && blockIdx.x < p.num_tiles) fetch_tile(row, tcol);
+        }
         if constexpr (DB) {
             if (is_fetcher && blockIdx.x + gridDim.x < p.num_tiles) {
                 int r1 = row, c1 = tcol;
@@ -800,6 +855,33 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             } else {
             if (is_fetcher && tile + (int)gridDim.x < p.num_tiles) fetch_tile(row_n, tcol_n);
             }
+        } else if constexpr (BSTG) {
+            if (!fk_wait_or_report(bar0, phase, p.wait_cycles, p.status)) return;
+            phase ^= 1u;
+            if (gB < gcount) {
+                const float2* bbase = reinterpret_cast<const float2*>(sStage0) + gB * P2;
+                auto load = [&](auto Kx) -> float2 {
+                    constexpr int kx = decltype(Kx)::value;
+                    // stored half: kx <= N/2; the other columns are mirror bins, conjugated
+                    auto fetch = [&](int ky) -> float2 {
+                        if (kx <= M) return bbase[ky * NC + kx];
+                        float2 t = bbase[((N - ky) & (N - 1)) * NC + (N - kx)];
+                        t.y = -t.y;
+                        return t;
+                    };
+                    float2 v = fetch(kyp);
+                    if (packed) {
+                        const float2 nq = fetch(M);
+                        v.x -= nq.y;
+                        v.y += nq.x;
+                    }
+                    return v;
+                };
+                if (q == 0) load_split<N, true, 0>(load, ar, ai);
+                else        load_split<N, true, 1>(load, ar, ai);
+            }
+            __syncthreads();        // planes in registers; previous tile's step 2 is done with sMid
+            if (is_fetcher && tile + (int)gridDim.x < p.num_tiles) fetch_bare(row_n, tcol_n);
         } else {
             if (gB < gcount) {
                 const size_t mat = (size_t)p.R * p.ld;
@@ -1008,11 +1090,10 @@ static bool fill_tiling(FftParams& p) {
 }
 
 // Forward transform of one operand, or of two operands in one launch (pb may be null).
-template <int N, bool FREQ>
-static cudaError_t launch_r2c_n(FftParams pa, const FftParams* pb_in, cudaStream_t st) {
+template <int N, int LAYOUT>
+static cudaError_t launch_r2c_layout(FftParams pa, const FftParams* pb_in, cudaStream_t st) {
     using Cfg = FftCfg<N>;
     constexpr int G = Cfg::G;
-    constexpr int LAYOUT = !FREQ ? LAYOUT_BARE : (Cfg::TMA ? LAYOUT_FREQ_TMA : LAYOUT_FREQ_DIRECT);
     FftParams pb{};
     if (!fill_tiling<G>(pa)) return cudaErrorInvalidValue;
     int in_bytes = real_tile_bytes(G, pa.h, pa.w);
@@ -1036,6 +1117,7 @@ static cudaError_t launch_r2c_n(FftParams pa, const FftParams* pb_in, cudaStream
         if (!make_spec_map<N, G>(&tma, pa.spec_out, pa)) return cudaErrorInvalidValue;
         if (pb_in && !make_spec_map<N, G>(&tmb, pb.spec_out, pb)) return cudaErrorInvalidValue;
     }
+    if (LAYOUT == LAYOUT_BARE_STAGED) smem += BareGeom<N, G>::BYTES;
     // the windowed variant (spatial tiling) is a separate instantiation, so that the plain
     // kernels carry none of its code
     const bool win = pa.win || (pb_in && pb.win);
@@ -1049,16 +1131,31 @@ static cudaError_t launch_r2c_n(FftParams pa, const FftParams* pb_in, cudaStream
     return dep_launch(false, kern, dim3(grid), dim3(N * G), smem, st, tma, tmb, pa, pb);
 }
 
+// Bare layout: staged through shared memory with bulk copies where a tile with its staging
+// image fits (n <= 64) and the spectrum is 16-byte aligned, else accessed by the threads.
+template <int N, bool FREQ>
+static cudaError_t launch_r2c_n(const FftParams& pa, const FftParams* pb_in, cudaStream_t st) {
+    using Cfg = FftCfg<N>;
+    if constexpr (FREQ) {
+        return launch_r2c_layout<N, Cfg::TMA ? LAYOUT_FREQ_TMA : LAYOUT_FREQ_DIRECT>(pa, pb_in, st);
+    } else {
+        if constexpr (N <= 64) {
+            if ((reinterpret_cast<uintptr_t>(pa.spec_out) & 15) == 0)
+                return launch_r2c_layout<N, LAYOUT_BARE_STAGED>(pa, pb_in, st);
+        }
+        return launch_r2c_layout<N, LAYOUT_BARE>(pa, pb_in, st);
+    }
+}
+
 // Plane sizes whose inverse transform double-buffers its staging tile.
 // Measured on B200: n = 64 (one resident CTA) 76-79 -> 72 us on the large-kernel layer, n = 16 44 -> 41 us
 // on the deep layer's accGrad; n = 32 loses a resident CTA to the second tile and gains nothing.
 template <int N> struct C2rDoubleBuffer { static constexpr bool value = (N == 64 || N == 16); };
 
-template <int N, bool FREQ>
-static cudaError_t launch_c2r_n(FftParams p, cudaStream_t st) {
+template <int N, int LAYOUT>
+static cudaError_t launch_c2r_layout(FftParams p, cudaStream_t st) {
     using Cfg = FftCfg<N>;
     constexpr int G = Cfg::G;
-    constexpr int LAYOUT = !FREQ ? LAYOUT_BARE : (Cfg::TMA ? LAYOUT_FREQ_TMA : LAYOUT_FREQ_DIRECT);
     constexpr bool DB = C2rDoubleBuffer<N>::value && LAYOUT == LAYOUT_FREQ_TMA;
     if (!fill_tiling<G>(p)) return cudaErrorInvalidValue;
     p.in_bytes = 0;
@@ -1069,6 +1166,7 @@ static cudaError_t launch_c2r_n(FftParams p, cudaStream_t st) {
         smem += (size_t)(DB ? 2 : 1) * 2 * N * (N / 2 + 1) * G * sizeof(float);
         if (!make_spec_map<N, G>(&tm, p.spec_in, p)) return cudaErrorInvalidValue;
     }
+    if (LAYOUT == LAYOUT_BARE_STAGED) smem += BareGeom<N, G>::BYTES;
     if (p.win && LAYOUT != LAYOUT_FREQ_TMA) return cudaErrorInvalidValue;
     auto kern = (p.win && LAYOUT == LAYOUT_FREQ_TMA) ? c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV, LAYOUT == LAYOUT_FREQ_TMA, DB>
                                                      : c2r_kernel<N, G, LAYOUT, Cfg::MINB_INV, false, DB>;
@@ -1076,6 +1174,20 @@ static cudaError_t launch_c2r_n(FftParams p, cudaStream_t st) {
     cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), N * G, smem, p.num_tiles, &grid);
     if (e != cudaSuccess) return e;
     return dep_launch(p.overlap != 0, kern, dim3(grid), dim3(N * G), smem, st, tm, p);
+}
+
+template <int N, bool FREQ>
+static cudaError_t launch_c2r_n(const FftParams& p, cudaStream_t st) {
+    using Cfg = FftCfg<N>;
+    if constexpr (FREQ) {
+        return launch_c2r_layout<N, Cfg::TMA ? LAYOUT_FREQ_TMA : LAYOUT_FREQ_DIRECT>(p, st);
+    } else {
+        if constexpr (N <= 64) {
+            if ((reinterpret_cast<uintptr_t>(p.spec_in) & 15) == 0)
+                return launch_c2r_layout<N, LAYOUT_BARE_STAGED>(p, st);
+        }
+        return launch_c2r_layout<N, LAYOUT_BARE>(p, st);
+    }
 }
 
 template <bool FREQ>

@@ -274,7 +274,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     bool forward_concurrent = false;
     auto forward_small = [&](const fc::FftParams& f, bool dep) -> cudaError_t {
         g_launches.fetch_add(1, std::memory_order_relaxed);
-        const bool conc = dep && !big && !timing && plan->small_planes == 1;
+        const bool conc = dep && !big && !timing;
         if (conc) forward_concurrent = true;
         return fc::launch_r2c_small(plan->n, f, 0, plan->n / 2 + 1, st, conc, conc);
     };
@@ -648,7 +648,7 @@ FFTCONV_API int conv_plan_set_filter_chunks(conv_plan_t* plan, int chunks) {
 
 FFTCONV_API int conv_plan_set_small_plane_kernel(conv_plan_t* plan, int enable) {
     if (!plan) return FFTCONV_EINVAL;
-    plan->small_planes = enable < 0 ? 0 : (enable > 2 ? 1 : enable);   // 2: without running beside the other transform (measurements)
+    plan->small_planes = enable ? 1 : 0;
     return FFTCONV_OK;
 }
 
