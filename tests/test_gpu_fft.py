@@ -115,3 +115,34 @@ def test_outputs_outside_the_result_are_untouched():
     torch.cuda.synchronize()
     assert torch.all(buf[:guard] == -7.25) and torch.all(buf[guard + nout:] == -7.25)
     assert not torch.any(out == -7.25)
+
+
+@pytest.mark.parametrize("n,batch,h,w", [(8, 37, 5, 3), (16, 70, 13, 13), (32, 35, 31, 31), (64, 9, 54, 33)])
+def test_bare_transforms_with_a_spectrum_that_is_only_8_byte_aligned(n, batch, h, w):
+    """A 16-byte-aligned spectrum travels by bulk copies through shared memory; one that is
+    only 8-byte aligned is accessed by the threads directly.  Both must give the same numbers."""
+    import torch
+    import oracle
+    import paper_1412_7580_b200 as fc
+    from paper_1412_7580_b200 import workloads as wl
+    x = wl.make_planes(batch, h, w, seed=n * 77 + w)
+    xd = torch.from_numpy(x).cuda()
+    nc = n // 2 + 1
+    buf = torch.full((batch * n * nc * 2 + 2,), float("nan"), device="cuda")
+    out = buf[2:].view(batch, n, nc, 2)                      # 8 bytes past a 16-byte boundary
+    assert out.data_ptr() % 16 == 8
+    fc.fft2d_r2c(xd, out, n)
+    aligned = torch.full((batch, n, nc, 2), float("nan"), device="cuda")
+    fc.fft2d_r2c(xd, aligned, n)
+    torch.cuda.synchronize()
+    assert torch.equal(out, aligned)
+    assert bool(torch.isnan(buf[:2]).all())                  # nothing written in front of the view
+    o = out.cpu().numpy().astype(np.float64)
+    assert relerr(o[..., 0] + 1j * o[..., 1], oracle.dft2d_r2c(x, n)) <= TOL_FFT
+    back_a = torch.full((batch, h, w), float("nan"), device="cuda")
+    back_u = torch.full((batch, h, w), float("nan"), device="cuda")
+    fc.fft2d_c2r(aligned, back_a, n, 1.0 / (n * n))
+    fc.fft2d_c2r(out, back_u, n, 1.0 / (n * n))
+    torch.cuda.synchronize()
+    assert torch.equal(back_a, back_u)
+    assert relerr(back_a.cpu().numpy().astype(np.float64), x.astype(np.float64)) <= TOL_FFT
