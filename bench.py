@@ -53,9 +53,44 @@ MAX_BLOCKS = 400
 # the bench reports the figure only while the sources still have that digest.
 NCU_TRAFFIC_SOURCE = {
     "profile": "profiles/dram_traffic_per_launch_three_layer_configs.md",
-    "kernel_sources_sha256": "unset",
+    "ncu": "dram__bytes_read.sum + dram__bytes_write.sum, default cache control (caches flushed before each launch)",
+    "kernel_sources_sha256": "d4fe69203e77caf2c193acda1e3d072453ecb84ad7b857f7634ea4d7f4caf510",
 }
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/fprop": 54.3e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/fprop": 46.8e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/fprop": 243.7e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/fprop": 193.4e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/bprop": 186.6e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/bprop": 46.9e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/bprop": 278.1e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/bprop": 54.8e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_both_operands/accgrad": 286.5e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/accgrad": 258.0e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/accgrad": 107.3e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/fprop": 227.0e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/fprop": 9.2e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/fprop": 289.5e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/fprop": 187.8e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/bprop": 183.3e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/bprop": 9.1e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/bprop": 289.5e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/bprop": 217.8e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_both_operands/accgrad": 457.4e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/accgrad": 324.2e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/accgrad": 69.6e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/fprop": 38.7e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/fprop": 114.1e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/fprop": 251.9e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/fprop": 56.7e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/bprop": 26.0e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/bprop": 113.6e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/bprop": 251.9e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/bprop": 56.8e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_both_operands/accgrad": 114.6e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/accgrad": 222.7e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/accgrad": 172.3e6,
+}
 
 
 def kernel_sources_digest():
@@ -310,6 +345,10 @@ class Bench:
         x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
         plan = fc.conv_plan(*s.args())
         fc.conv_plan_set_math(plan, math)
+        if args.filter_chunks > 1:
+            fc.conv_plan_set_filter_chunks(plan, args.filter_chunks)
+        if args.no_small_planes:
+            fc.conv_plan_set_small_plane_kernel(plan, False)
         if tile_req:
             fc.conv_plan_set_tiling(plan, tile_req)      # -1: the plan chooses
         tile = fc.conv_plan_tile_basis(plan)
@@ -654,7 +693,8 @@ def run_ours(args):
     from paper_1412_7580_b200 import workloads as wl
     b = Bench(args)
     math = {"auto": fc.MATH_AUTO, "fp32": fc.MATH_FP32, "tf32": fc.MATH_TF32}[args.math]
-    single = args.config is not None or args.shape is not None
+    single = (args.config is not None or args.shape is not None or args.filter_chunks > 1
+              or args.no_small_planes)
     extras = not single and not args.no_extras and b.world == 1
 
     if args.fft2d or args.fft1d:
@@ -728,6 +768,10 @@ def main():
     ap.add_argument("--tile", type=int, default=0,
                     help="spatial tiling with this basis (8, 16, 32 or 64; 0 = off); bytes, flops and the "
                          "roofline in the output are then those of the tiled method")
+    ap.add_argument("--filter-chunks", type=int, default=1,
+                    help="fprop / bprop: transform and contract the filters in this many ranges of frequency rows")
+    ap.add_argument("--no-small-planes", action="store_true",
+                    help="send the filters through the butterfly kernels instead of the small-plane kernel")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-reuse-line", action="store_true",

@@ -8,7 +8,8 @@
 // C is [2][bins][M][ldc].
 //
 // CTA tile 64 x 64 of one bin, 256 threads, each thread a 4 x 4 block of complex
-// outputs (64 FFMAs per k against four 16-byte shared loads).  This is the exact
+// outputs (64 FFMAs per k against four 16-byte shared loads); k-blocks of 16 arrive by
+// asynchronous copies, double-buffered.  This is the exact
 // fp32 path and the fallback for shapes too small for the tensor-core kernel.
 #pragma once
 
@@ -36,9 +37,21 @@ struct GemmParams {
 
 constexpr int FG_BM = 64, FG_BN = 64, FG_BK = 16, FG_PAD = 4, FG_T = 256;
 
+// 4-byte asynchronous copy global -> shared; `ok` false writes a zero (zero-fill of the
+// ragged edges of M, N and K).
+__device__ __forceinline__ void fg_cp4(float* dst, const float* src, bool ok) {
+    const unsigned d = static_cast<unsigned>(__cvta_generic_to_shared(dst));
+    const int nbytes = ok ? 4 : 0;
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(d), "l"(src), "r"(nbytes) : "memory");
+}
+
+// TA / TB: operand stored [K][rows] instead of [rows][K]; CA / CB: use its complex conjugate.
+// The k-blocks are double-buffered in shared memory: the asynchronous copies of block kb + 1
+// are in flight while block kb is multiplied.
+template <bool TA, bool TB, bool CA, bool CB>
 __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
-    __shared__ __align__(16) float sA[2][FG_BK][FG_BM + FG_PAD];
-    __shared__ __align__(16) float sB[2][FG_BK][FG_BN + FG_PAD];
+    __shared__ __align__(16) float sA[2][2][FG_BK][FG_BM + FG_PAD];
+    __shared__ __align__(16) float sB[2][2][FG_BK][FG_BN + FG_PAD];
 
     dep_trigger();
     dep_wait();                     // no global access above this line
@@ -48,9 +61,8 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
     const int bin = blockIdx.y;
     const int n_blocks = (p.N + FG_BN - 1) / FG_BN;
     const int m_blk = (int)(blockIdx.x / n_blocks) * FG_BM, n_blk = (int)(blockIdx.x % n_blocks) * FG_BN;
-    const size_t planeA = (size_t)(p.transA ? p.K : p.M) * p.lda,
-                 planeB = (size_t)(p.transB ? p.K : p.N) * p.ldb, planeC = (size_t)p.M * p.ldc;
-    const float sa = p.conjA ? -1.0f : 1.0f, sb = p.conjB ? -1.0f : 1.0f;
+    const size_t planeA = (size_t)(TA ? p.K : p.M) * p.lda,
+                 planeB = (size_t)(TB ? p.K : p.N) * p.ldb, planeC = (size_t)p.M * p.ldc;
     const float* Ab = p.A + (size_t)bin * planeA;
     const float* Bb = p.B + (size_t)bin * planeB;
     float* Cb = p.C + (size_t)bin * planeC;
@@ -58,7 +70,55 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
                  imC = (size_t)p.bins * planeC;
 
     const int tx = tid & 15, ty = tid >> 4;      // 16 x 16 threads
-    const int lk = tid & 15, lr = tid >> 4;      // loader: k within chunk, row group
+    const int lk = tid & 15, lr = tid >> 4;      // loader, k-contiguous operand: k within block, row group
+    const int tr = tid & 63, tk = tid >> 6;      // loader, row-contiguous operand: row, k group
+
+    // global -> shared as [k][row]; lanes run along the contiguous index of each operand
+    auto issue = [&](int k0, int st) {
+        if constexpr (!TA) {
+            const int k = k0 + lk;
+#pragma unroll
+            for (int it = 0; it < FG_BM / 16; ++it) {
+                const int r = lr + 16 * it, m = m_blk + r;
+                const bool ok = (k < p.K) && (m < p.M);
+                const float* src = ok ? Ab + (size_t)m * p.lda + k : Ab;
+                fg_cp4(&sA[st][0][lk][r], src, ok);
+                fg_cp4(&sA[st][1][lk][r], src + imA, ok);
+            }
+        } else {
+            const int m = m_blk + tr;
+#pragma unroll
+            for (int it = 0; it < FG_BK / 4; ++it) {
+                const int kk = tk + 4 * it, k = k0 + kk;
+                const bool ok = (k < p.K) && (m < p.M);
+                const float* src = ok ? Ab + (size_t)k * p.lda + m : Ab;
+                fg_cp4(&sA[st][0][kk][tr], src, ok);
+                fg_cp4(&sA[st][1][kk][tr], src + imA, ok);
+            }
+        }
+        if constexpr (!TB) {
+            const int k = k0 + lk;
+#pragma unroll
+            for (int it = 0; it < FG_BN / 16; ++it) {
+                const int r = lr + 16 * it, n = n_blk + r;
+                const bool ok = (k < p.K) && (n < p.N);
+                const float* src = ok ? Bb + (size_t)n * p.ldb + k : Bb;
+                fg_cp4(&sB[st][0][lk][r], src, ok);
+                fg_cp4(&sB[st][1][lk][r], src + imB, ok);
+            }
+        } else {
+            const int n = n_blk + tr;
+#pragma unroll
+            for (int it = 0; it < FG_BK / 4; ++it) {
+                const int kk = tk + 4 * it, k = k0 + kk;
+                const bool ok = (k < p.K) && (n < p.N);
+                const float* src = ok ? Bb + (size_t)k * p.ldb + n : Bb;
+                fg_cp4(&sB[st][0][kk][tr], src, ok);
+                fg_cp4(&sB[st][1][kk][tr], src + imB, ok);
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
 
     float cr[4][4], ci[4][4];
 #pragma unroll
@@ -66,81 +126,40 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) cr[i][j] = ci[i][j] = 0.0f;
 
-    for (int k0 = 0; k0 < p.K; k0 += FG_BK) {
-        // global -> shared as [k][row]; zero-fill outside M/N/K; lanes run along the
-        // contiguous index of each operand
-        if (!p.transA) {
-            const int k = k0 + lk;
-#pragma unroll
-            for (int it = 0; it < FG_BM / 16; ++it) {
-                const int r = lr + 16 * it, m = m_blk + r;
-                float are = 0.f, aim = 0.f;
-                if (k < p.K && m < p.M) {
-                    are = __ldg(Ab + (size_t)m * p.lda + k);
-                    aim = sa * __ldg(Ab + imA + (size_t)m * p.lda + k);
-                }
-                sA[0][lk][r] = are; sA[1][lk][r] = aim;
-            }
+    const int k_blocks = (p.K + FG_BK - 1) / FG_BK;
+    issue(0, 0);
+    for (int kb = 0; kb < k_blocks; ++kb) {
+        const int st = kb & 1;
+        if (kb + 1 < k_blocks) {
+            issue((kb + 1) * FG_BK, st ^ 1);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");    // block kb has landed (for this thread)
         } else {
-            const int r = tid & 63, m = m_blk + r;
-#pragma unroll
-            for (int it = 0; it < FG_BK / 4; ++it) {
-                const int kk = (tid >> 6) + 4 * it, k = k0 + kk;
-                float are = 0.f, aim = 0.f;
-                if (k < p.K && m < p.M) {
-                    are = __ldg(Ab + (size_t)k * p.lda + m);
-                    aim = sa * __ldg(Ab + imA + (size_t)k * p.lda + m);
-                }
-                sA[0][kk][r] = are; sA[1][kk][r] = aim;
-            }
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
         }
-        if (!p.transB) {
-            const int k = k0 + lk;
-#pragma unroll
-            for (int it = 0; it < FG_BN / 16; ++it) {
-                const int r = lr + 16 * it, n = n_blk + r;
-                float bre = 0.f, bim = 0.f;
-                if (k < p.K && n < p.N) {
-                    bre = __ldg(Bb + (size_t)n * p.ldb + k);
-                    bim = sb * __ldg(Bb + imB + (size_t)n * p.ldb + k);
-                }
-                sB[0][lk][r] = bre; sB[1][lk][r] = bim;
-            }
-        } else {
-            const int r = tid & 63, n = n_blk + r;
-#pragma unroll
-            for (int it = 0; it < FG_BK / 4; ++it) {
-                const int kk = (tid >> 6) + 4 * it, k = k0 + kk;
-                float bre = 0.f, bim = 0.f;
-                if (k < p.K && n < p.N) {
-                    bre = __ldg(Bb + (size_t)k * p.ldb + n);
-                    bim = sb * __ldg(Bb + imB + (size_t)k * p.ldb + n);
-                }
-                sB[0][kk][r] = bre; sB[1][kk][r] = bim;
-            }
-        }
-        __syncthreads();
+        __syncthreads();                                            // ... and for everyone
 #pragma unroll
         for (int kk = 0; kk < FG_BK; ++kk) {
-            const float4 a_r = *reinterpret_cast<const float4*>(&sA[0][kk][ty * 4]);
-            const float4 a_i = *reinterpret_cast<const float4*>(&sA[1][kk][ty * 4]);
-            const float4 b_r = *reinterpret_cast<const float4*>(&sB[0][kk][tx * 4]);
-            const float4 b_i = *reinterpret_cast<const float4*>(&sB[1][kk][tx * 4]);
+            const float4 a_r = *reinterpret_cast<const float4*>(&sA[st][0][kk][ty * 4]);
+            const float4 a_i = *reinterpret_cast<const float4*>(&sA[st][1][kk][ty * 4]);
+            const float4 b_r = *reinterpret_cast<const float4*>(&sB[st][0][kk][tx * 4]);
+            const float4 b_i = *reinterpret_cast<const float4*>(&sB[st][1][kk][tx * 4]);
             const float ar[4] = {a_r.x, a_r.y, a_r.z, a_r.w};
             const float ai[4] = {a_i.x, a_i.y, a_i.z, a_i.w};
             const float br[4] = {b_r.x, b_r.y, b_r.z, b_r.w};
             const float bi[4] = {b_i.x, b_i.y, b_i.z, b_i.w};
+            // (ar + i sa ai)(br + i sb bi), sa / sb = -1 for a conjugated operand:
+            // re = ar br - sa sb ai bi,  im = sb ar bi + sa ai br
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     cr[i][j] = fmaf(ar[i], br[j], cr[i][j]);
-                    cr[i][j] = fmaf(-ai[i], bi[j], cr[i][j]);
-                    ci[i][j] = fmaf(ar[i], bi[j], ci[i][j]);
-                    ci[i][j] = fmaf(ai[i], br[j], ci[i][j]);
+                    cr[i][j] = fmaf((CA != CB) ? ai[i] : -ai[i], bi[j], cr[i][j]);
+                    ci[i][j] = fmaf(CB ? -ar[i] : ar[i], bi[j], ci[i][j]);
+                    ci[i][j] = fmaf(CA ? -ai[i] : ai[i], br[j], ci[i][j]);
                 }
         }
-        __syncthreads();
+        __syncthreads();                                            // stage st may be refilled
     }
 
     const int n0 = n_blk + tx * 4;
@@ -161,11 +180,21 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
     }
 }
 
+template <bool TA, bool TB>
+static cudaError_t launch_cgemm_ffma_t(const GemmParams& p, dim3 grid, cudaStream_t st) {
+    const bool ov = p.overlap != 0;
+    if (p.conjA) return p.conjB ? dep_launch(ov, cgemm_ffma_kernel<TA, TB, true, true>, grid, dim3(FG_T), 0, st, p)
+                                : dep_launch(ov, cgemm_ffma_kernel<TA, TB, true, false>, grid, dim3(FG_T), 0, st, p);
+    return p.conjB ? dep_launch(ov, cgemm_ffma_kernel<TA, TB, false, true>, grid, dim3(FG_T), 0, st, p)
+                   : dep_launch(ov, cgemm_ffma_kernel<TA, TB, false, false>, grid, dim3(FG_T), 0, st, p);
+}
+
 static cudaError_t launch_cgemm_ffma(const GemmParams& p, cudaStream_t st) {
     const long long blocks = (long long)((p.N + FG_BN - 1) / FG_BN) * ((p.M + FG_BM - 1) / FG_BM);
     if (blocks > 0x7fffffffLL || p.bins > 65535) return cudaErrorInvalidValue;
     dim3 grid((unsigned)blocks, (unsigned)p.bins, 1);
-    return dep_launch(p.overlap != 0, cgemm_ffma_kernel, grid, dim3(FG_T), 0, st, p);
+    if (p.transA) return p.transB ? launch_cgemm_ffma_t<true, true>(p, grid, st) : launch_cgemm_ffma_t<true, false>(p, grid, st);
+    return p.transB ? launch_cgemm_ffma_t<false, true>(p, grid, st) : launch_cgemm_ffma_t<false, false>(p, grid, st);
 }
 
 }  // namespace fc

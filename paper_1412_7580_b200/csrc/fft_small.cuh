@@ -77,8 +77,10 @@ r2c_small_kernel(const SmallParams p) {
 
     dep_trigger();
     // `concurrent`: the predecessor in the stream is the other operand's forward transform, which
-    // this kernel neither reads from nor overwrites; the launch that follows both is a plain one
-    // and therefore waits for both.
+    // this kernel neither reads from nor overwrites, so it does not wait for it before it starts.
+    // It waits for it at its END instead (below): this grid then completes only after its
+    // predecessor has, and the kernel launched after it as a programmatic dependent, which waits
+    // for this grid alone, is ordered after both.
     if (!p.concurrent) dep_wait();  // no global access above this line
 
     const long long stride = (long long)gridDim.x * SMALL_WARPS;
@@ -171,6 +173,7 @@ r2c_small_kernel(const SmallParams p) {
             });
         }
     }
+    if (p.concurrent) dep_wait();   // see above: complete only after the predecessor has
 }
 
 // True if the small-plane kernel takes this operand: planes that fill at most a quarter of
@@ -214,8 +217,8 @@ static cudaError_t launch_r2c_small_n(const SmallParams& p, cudaStream_t st, boo
 // Forward transform of one operand whose planes are small (see small_supported); produces the
 // rows ky in [ky_begin, ky_end) of the kept half, all kx.
 // overlap: launch as a programmatic dependent of the previous kernel.  concurrent (with overlap):
-// additionally skip the wait for that kernel, so that the two run side by side; the caller must
-// then launch the next kernel the plain way (a plain launch waits for everything before it).
+// additionally start without waiting for that kernel, so that the two run side by side (the wait
+// moves to the end of this kernel, which keeps the chain of dependent launches ordered).
 static cudaError_t launch_r2c_small(int n, const FftParams& f, int ky_begin, int ky_end, cudaStream_t st,
                                     bool overlap = false, bool concurrent = false) {
     if (!small_supported(n, f.h, f.w) || f.win) return cudaErrorNotSupported;

@@ -269,13 +269,10 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         return plan->small_planes && !f.win && fc::small_supported(plan->n, f.h, f.w);
     };
     // dep: another forward transform of this pass was launched just before; the small-plane kernel
-    // then runs beside it (neither touches the other's data) and the contraction is launched the
-    // plain way, which waits for both.
-    bool forward_concurrent = false;
+    // then runs beside it (neither touches the other's data) and completes only after it.
     auto forward_small = [&](const fc::FftParams& f, bool dep) -> cudaError_t {
         g_launches.fetch_add(1, std::memory_order_relaxed);
         const bool conc = dep && !big && !timing;
-        if (conc) forward_concurrent = true;
         return fc::launch_r2c_small(plan->n, f, 0, plan->n / 2 + 1, st, conc, conc);
     };
     mark(0);
@@ -340,8 +337,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         plan->cached[d.b.kind] = b_in;
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    // predecessor: this pass's forward transforms (plain launch after two that ran side by side)
-    gp.overlap = (overlap && (need_a || need_b) && !forward_concurrent) ? 1 : 0;
+    gp.overlap = (overlap && (need_a || need_b)) ? 1 : 0;       // predecessor: this pass's forward transforms
     cudaError_t ge;
     if (tensor) ge = fc::launch_cgemm_tc(gp, status, st);
     else ge = fc::launch_cgemm_ffma(gp, st);
