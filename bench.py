@@ -54,41 +54,41 @@ MAX_BLOCKS = 400
 NCU_TRAFFIC_SOURCE = {
     "profile": "profiles/dram_traffic_per_launch_three_layer_configs.md",
     "ncu": "dram__bytes_read.sum + dram__bytes_write.sum, default cache control (caches flushed before each launch)",
-    "kernel_sources_sha256": "d4fe69203e77caf2c193acda1e3d072453ecb84ad7b857f7634ea4d7f4caf510",
+    "kernel_sources_sha256": "e3bedc00e3b1be5c71b75181f53ca68ab4a4481c262c8544a1b0509e2fae7668",
 }
 NCU_TRAFFIC = {
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/fprop": 54.3e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/fprop": 46.8e6,
-    "mid_S128_f96_fp256_31x31_k5/bin_contraction/fprop": 243.7e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/fprop": 193.4e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/bprop": 186.6e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/bprop": 46.9e6,
-    "mid_S128_f96_fp256_31x31_k5/bin_contraction/bprop": 278.1e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/bprop": 54.8e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_both_operands/accgrad": 286.5e6,
-    "mid_S128_f96_fp256_31x31_k5/bin_contraction/accgrad": 258.0e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/fprop": 54.0e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/fprop": 46.3e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/fprop": 242.4e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/fprop": 193.7e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/bprop": 186.3e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/bprop": 46.8e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/bprop": 277.6e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/bprop": 54.4e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_both_operands/accgrad": 286.7e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/accgrad": 258.2e6,
     "mid_S128_f96_fp256_31x31_k5/c2r_ifft/accgrad": 107.3e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/fprop": 227.0e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/fprop": 226.8e6,
     "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/fprop": 9.2e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/fprop": 289.5e6,
-    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/fprop": 187.8e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/bprop": 183.3e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/bprop": 9.1e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/bprop": 289.5e6,
-    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/bprop": 217.8e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_both_operands/accgrad": 457.4e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/accgrad": 324.2e6,
-    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/accgrad": 69.6e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/fprop": 38.7e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/fprop": 114.1e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/fprop": 289.4e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/fprop": 187.9e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/bprop": 182.9e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/bprop": 9.2e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/bprop": 290.2e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/bprop": 217.2e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_both_operands/accgrad": 457.5e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/accgrad": 324.0e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/accgrad": 69.3e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/fprop": 38.6e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/fprop": 113.9e6,
     "deep_S128_f384_fp384_13x13_k3/bin_contraction/fprop": 251.9e6,
     "deep_S128_f384_fp384_13x13_k3/c2r_ifft/fprop": 56.7e6,
     "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/bprop": 26.0e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/bprop": 113.6e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/bprop": 113.5e6,
     "deep_S128_f384_fp384_13x13_k3/bin_contraction/bprop": 251.9e6,
-    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/bprop": 56.8e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/bprop": 56.7e6,
     "deep_S128_f384_fp384_13x13_k3/r2c_fft_both_operands/accgrad": 114.6e6,
-    "deep_S128_f384_fp384_13x13_k3/bin_contraction/accgrad": 222.7e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/accgrad": 222.8e6,
     "deep_S128_f384_fp384_13x13_k3/c2r_ifft/accgrad": 172.3e6,
 }
 
