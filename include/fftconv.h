@@ -89,8 +89,10 @@ size_t conv_plan_workspace_bytes(const conv_plan_t* plan);
 /* Lend the plan `bytes` of device memory at `dev_ptr` (256-byte aligned).  The
  * caller keeps ownership and must keep it alive while the plan is used.
  * Contents need no initialisation and are overwritten by every pass.  Passes of
- * one plan must not overlap in time (one workspace).  EWORKSPACE if too small
- * or misaligned. */
+ * one plan must not overlap in time (one workspace).  The call clears the
+ * 256-byte header in front of the spectra (the device status word lives there)
+ * with a synchronous cudaMemset: it is a set-up call, not for the hot loop.
+ * EWORKSPACE if too small or misaligned. */
 int conv_plan_set_workspace(conv_plan_t* plan, void* dev_ptr, size_t bytes);
 
 /* fprop (Section 2, first equation): y(s,j) = sum_i x(s,i) (star) w(j,i), valid
@@ -137,13 +139,17 @@ int conv_bprop(conv_plan_t* plan, const float* dy, const float* w, float* dx, vo
 int conv_accgrad(conv_plan_t* plan, const float* dy, const float* x, float* dw, int accumulate,
                  void* cuda_stream);
 
-/* Forward transform of small planes.  Operand planes of at most 13 x 13 samples (the filters
- * of fprop and bprop) are transformed by a pruned separable DFT that evaluates one frequency
- * bin for 32 adjacent planes at a time and writes whole 128-byte lines of the frequency-major
- * spectrum (Section 5.1: the padding is never materialised -- here it is never even
- * multiplied), instead of by the butterfly kernels that the large planes use.  On by default;
- * enable == 0 sends every operand through the butterfly kernels (same results up to
- * rounding).  The operand then has a launch of its own: a pass is four launches. */
+/* Transforms of small planes.  Operand planes of at most 13 x 13 samples that fill at most a
+ * quarter of the basis (the filters of fprop and bprop) are transformed by a pruned separable
+ * DFT that evaluates one frequency bin for 32 adjacent planes at a time and writes whole
+ * 128-byte lines of the frequency-major spectrum (Section 5.1: the padding is never
+ * materialised -- here it is never even multiplied), instead of by the butterfly kernels that
+ * the large planes use; the operand then has a launch of its own, which runs beside the other
+ * operand's transform (a pass is four launches).  Likewise the inverse transform of accGrad,
+ * whose result is clipped to the kh x kw filter window (Section 3.1), is a pruned inverse DFT
+ * that reads whole lines for 32 adjacent planes when the window is square, at most 11 x 11 and
+ * at most a quarter of the basis (n = 32 and 64).  On by default; enable == 0 sends everything
+ * through the butterfly kernels (same results up to rounding). */
 int conv_plan_set_small_plane_kernel(conv_plan_t* plan, int enable);
 
 /* Filter spectrum through the cache (Section 6 asks for fewer passes over memory between the

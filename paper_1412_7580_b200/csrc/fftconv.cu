@@ -356,9 +356,13 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     ip.overlap = overlap ? 1 : 0;
     ip.status = status; ip.wait_cycles = plan->wait_cycles;
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    if ((big ? fc::launch_c2r_two_pass(plan->n, ip, scratch, scratch_bytes, st)
-             : fc::launch_c2r<true>(plan->n, ip, st)) != cudaSuccess)
-        return FFTCONV_ECUDA;
+    // a small square crop (the filter gradient of accGrad) takes the pruned inverse kernel,
+    // whose loads are whole 128-byte lines; everything else the butterfly kernels
+    cudaError_t ie = plan->small_planes ? fc::launch_c2r_small(plan->n, ip, st) : cudaErrorNotSupported;
+    if (ie == cudaErrorNotSupported)
+        ie = big ? fc::launch_c2r_two_pass(plan->n, ip, scratch, scratch_bytes, st)
+                 : fc::launch_c2r<true>(plan->n, ip, st);
+    if (ie != cudaSuccess) return FFTCONV_ECUDA;
     mark(4);
     if (timing) plan->timed = true;
     return FFTCONV_OK;

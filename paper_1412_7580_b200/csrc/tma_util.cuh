@@ -6,6 +6,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 namespace fc {
 
 typedef CUresult (*tc_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
@@ -13,18 +15,22 @@ typedef CUresult (*tc_encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, 
                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// The entry point is the same for every device and thread: looked up once, published
+// through an atomic (concurrent first calls all store the same pointer).
 static tc_encode_fn tc_get_encode() {
-    static tc_encode_fn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* sym = nullptr;
+    static std::atomic<void*> cached{nullptr};
+    static std::atomic<bool> tried{false};
+    void* sym = cached.load(std::memory_order_acquire);
+    if (!sym && !tried.load(std::memory_order_acquire)) {
         cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) ==
+        void* found = nullptr;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &found, cudaEnableDefault, &qres) ==
                 cudaSuccess && qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<tc_encode_fn>(sym);
+            sym = found;
+        cached.store(sym, std::memory_order_release);
+        tried.store(true, std::memory_order_release);
     }
-    return fn;
+    return reinterpret_cast<tc_encode_fn>(sym);
 }
 
 // Planar matrix family [2][bins][rows][ld] (all real matrices, then all imaginary
