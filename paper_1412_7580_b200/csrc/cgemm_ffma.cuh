@@ -33,6 +33,10 @@ struct GemmParams {
     // with ky_count > 0 only the rows ky in [ky_begin, ky_begin + ky_count) of every kx are
     // contracted (bins / nc values of kx).  ky_count == 0: all bins.
     int nc, ky_begin, ky_count;
+    // Tensor-core kernel only, host only: the next launch in the stream is a transform that is to
+    // run beside this contraction; the kernel then keeps 64 KB of shared memory free (two pipeline
+    // stages instead of three) and releases its dependent only after its own wait.
+    int shared_sms;
 };
 
 constexpr int FG_BM = 64, FG_BN = 64, FG_BK = 16, FG_PAD = 4, FG_T = 256;

@@ -49,7 +49,11 @@ constexpr uint32_t TC_TILE_BYTES = TC_BM * TC_BK * 4;            // one 128 x 32
 constexpr uint32_t TC_STAGE_BYTES = 4 * TC_TILE_BYTES;           // A_re, A_im, B_re, B_im
 constexpr uint32_t TC_EPI_BUF_BYTES = 32 * 128;                  // 32 rows x 32 fp32, one TMA store box
 constexpr uint32_t TC_EPI_BYTES = 4 * 2 * TC_EPI_BUF_BYTES;      // 4 warps x 2 buffers
-constexpr uint32_t TC_SMEM_BYTES = 1024 + TC_STAGES * TC_STAGE_BYTES + TC_EPI_BYTES + 256;
+constexpr uint32_t tc_smem_bytes(int stages) { return 1024 + stages * TC_STAGE_BYTES + TC_EPI_BYTES + 256; }
+constexpr uint32_t TC_SMEM_BYTES = tc_smem_bytes(TC_STAGES);
+// A launch that shares the SMs with a transform kernel (the filter spectrum produced range by range
+// beside the contraction) runs a ring of two stages and leaves 64 KB of shared memory to that kernel.
+constexpr int TC_STAGES_SHARED = 2;
 constexpr uint32_t TC_TMEM_COLS = 512;
 constexpr long long TC_WAIT_CYCLES = 2000000000LL;               // about one second
 
@@ -61,6 +65,7 @@ struct TcParams {
     long long wait_cycles;      // limit of one wait in SM clock cycles (the draining waits keep TC_WAIT_CYCLES)
     int bins_run;               // bins contracted by this launch (all of them, or a ky range of every kx)
     int nc, ky_begin, ky_count; // ky_count > 0: local bin b -> kx = b / ky_count, ky = ky_begin + b % ky_count
+    int late_trigger;           // let the dependent launch start after this one's wait instead of before it
 };
 
 static inline bool tc_shape_supported(int M, int N, int K) {
@@ -189,30 +194,30 @@ __host__ __device__ constexpr uint32_t tc_idesc(int M, int N, bool negA, bool mn
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
-template <bool TA, bool TB>
+template <bool TA, bool TB, int ST>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                 const __grid_constant__ CUtensorMap tmC, const TcParams p) {
     extern __shared__ uint8_t tc_raw[];
     const uint32_t raw_addr = smem_u32(tc_raw);
     const uint32_t tiles = (raw_addr + 1023u) & ~1023u;             // stage buffers, 1024-aligned
-    const uint32_t epi = tiles + TC_STAGES * TC_STAGE_BYTES;        // epilogue staging, 1024-aligned
-    uint8_t* ctl = tc_raw + (tiles - raw_addr) + TC_STAGES * TC_STAGE_BYTES + TC_EPI_BYTES;
+    const uint32_t epi = tiles + ST * TC_STAGE_BYTES;        // epilogue staging, 1024-aligned
+    uint8_t* ctl = tc_raw + (tiles - raw_addr) + ST * TC_STAGE_BYTES + TC_EPI_BYTES;
     const uint32_t bars = epi + TC_EPI_BYTES;
     // barrier slots (8 bytes each): full[3] empty[3] tfull[2] tempty[2] drain
     auto full = [&](int s) { return bars + 8u * s; };
-    auto empty = [&](int s) { return bars + 8u * (TC_STAGES + s); };
-    auto tfull = [&](int b) { return bars + 8u * (2 * TC_STAGES + b); };
-    auto tempty = [&](int b) { return bars + 8u * (2 * TC_STAGES + 2 + b); };
-    const uint32_t drain = bars + 8u * (2 * TC_STAGES + 4);
+    auto empty = [&](int s) { return bars + 8u * (ST + s); };
+    auto tfull = [&](int b) { return bars + 8u * (2 * ST + b); };
+    auto tempty = [&](int b) { return bars + 8u * (2 * ST + 2 + b); };
+    const uint32_t drain = bars + 8u * (2 * ST + 4);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + 128);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + 136);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-    dep_trigger();
+    if (!p.late_trigger) dep_trigger();
     if (tid == 0) {
-        for (int s = 0; s < TC_STAGES; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
+        for (int s = 0; s < ST; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(tfull(b), 1); mbar_init(tempty(b), 128); }
         mbar_init(drain, 1);
         *abort_flag = 0;
@@ -228,6 +233,9 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     dep_wait();                     // no global access above this line
+    // late: the dependent is a transform that runs beside this contraction (not after it) and
+    // must not start before the operands of this launch are complete
+    if (p.late_trigger) dep_trigger();
 
     const int num_tiles = p.bins_run * p.m_tiles * p.n_tiles;
     // local bin of this launch -> bin of the spectra
@@ -251,8 +259,8 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const int m_t = (t / p.n_tiles) % p.m_tiles;
                 const int bin = global_bin(t / (p.n_tiles * p.m_tiles));
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % TC_STAGES;
-                    const uint32_t ph = (uint32_t)(it / TC_STAGES) & 1u;
+                    const int s = it % ST;
+                    const uint32_t ph = (uint32_t)(it / ST) & 1u;
                     if (!mbar_wait(empty(s), ph ^ 1u, abort_flag, p.wait_cycles)) { ok = false; break; }
                     const uint32_t dst = tiles + s * TC_STAGE_BYTES;
                     mbar_expect_tx(full(s), TC_STAGE_BYTES);
@@ -282,10 +290,10 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             if (!ok) {
                 give_up();
                 // let the copies already issued land before the CTA's memory goes away
-                const int back = it < TC_STAGES ? it : TC_STAGES;
+                const int back = it < ST ? it : ST;
                 for (int j = it - back; j < it; ++j) {
                     const long long t0 = clock64();
-                    while (!mbar_try_wait(full(j % TC_STAGES), (uint32_t)(j / TC_STAGES) & 1u) &&
+                    while (!mbar_try_wait(full(j % ST), (uint32_t)(j / ST) & 1u) &&
                            clock64() - t0 < TC_WAIT_CYCLES) {}
                 }
             }
@@ -308,8 +316,8 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 const uint32_t d_re = tmem_base + (uint32_t)buf * 256u;
                 const uint32_t d_im = d_re + 128u;
                 for (int kb = 0; kb < p.k_blocks; ++kb, ++it) {
-                    const int s = it % TC_STAGES;
-                    if (!mbar_wait(full(s), (uint32_t)(it / TC_STAGES) & 1u, abort_flag, p.wait_cycles)) { ok = false; break; }
+                    const int s = it % ST;
+                    if (!mbar_wait(full(s), (uint32_t)(it / ST) & 1u, abort_flag, p.wait_cycles)) { ok = false; break; }
                     tc_fence_after_sync();
                     const uint32_t src = tiles + s * TC_STAGE_BYTES;
                     const uint64_t a_re = TA ? tc_smem_desc_mn(src) : tc_smem_desc(src);
@@ -408,15 +416,15 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
 }
 
 // ---- host side -------------------------------------------------------------
-template <bool TA, bool TB>
+template <bool TA, bool TB, int ST>
 static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStream_t st, int sm_count) {
-    auto kern = cgemm_tc_kernel<TA, TB>;
+    auto kern = cgemm_tc_kernel<TA, TB, ST>;
     static std::atomic<unsigned long long> attr_set_devices{0};     // one bit per device ordinal
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
     if (dev < 0 || dev >= 64 || !((attr_set_devices.load(std::memory_order_acquire) >> dev) & 1ull)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)TC_SMEM_BYTES);
+                                             (int)tc_smem_bytes(ST));
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set_devices.fetch_or(1ull << dev, std::memory_order_release);
     }
@@ -440,6 +448,7 @@ static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStrea
     p.status = status;
     p.wait_cycles = g.wait_cycles > 0 ? g.wait_cycles : TC_WAIT_CYCLES;
     p.bins_run = g.bins; p.nc = g.nc; p.ky_begin = g.ky_begin; p.ky_count = 0;
+    p.late_trigger = g.shared_sms ? 1 : 0;
     if (g.ky_count > 0) {
         if (g.nc < 1 || g.bins % g.nc != 0 || g.ky_begin < 0 || g.ky_begin + g.ky_count > g.nc)
             return cudaErrorInvalidValue;
@@ -448,16 +457,23 @@ static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStrea
     const long long tiles = (long long)p.bins_run * p.m_tiles * p.n_tiles;
     if (tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
     const int grid = (int)(tiles < sm_count ? tiles : sm_count);
-    return dep_launch(g.overlap != 0, kern, dim3(grid), dim3(TC_THREADS), TC_SMEM_BYTES, st, tmA, tmB, tmC, p);
+    return dep_launch(g.overlap != 0, kern, dim3(grid), dim3(TC_THREADS), tc_smem_bytes(ST), st, tmA, tmB, tmC, p);
 }
 
 static cudaError_t launch_cgemm_tc(const GemmParams& g, int* status, cudaStream_t st) {
     const int sm_count = fft_sm_count();        // of the current device
     if (sm_count < 1) return cudaErrorInvalidDevice;
-    if (g.transA) return g.transB ? launch_cgemm_tc_t<true, true>(g, status, st, sm_count)
-                                  : launch_cgemm_tc_t<true, false>(g, status, st, sm_count);
-    return g.transB ? launch_cgemm_tc_t<false, true>(g, status, st, sm_count)
-                    : launch_cgemm_tc_t<false, false>(g, status, st, sm_count);
+    if (g.shared_sms) {
+        constexpr int S2 = TC_STAGES_SHARED;
+        if (g.transA) return g.transB ? launch_cgemm_tc_t<true, true, S2>(g, status, st, sm_count)
+                                      : launch_cgemm_tc_t<true, false, S2>(g, status, st, sm_count);
+        return g.transB ? launch_cgemm_tc_t<false, true, S2>(g, status, st, sm_count)
+                        : launch_cgemm_tc_t<false, false, S2>(g, status, st, sm_count);
+    }
+    if (g.transA) return g.transB ? launch_cgemm_tc_t<true, true, TC_STAGES>(g, status, st, sm_count)
+                                  : launch_cgemm_tc_t<true, false, TC_STAGES>(g, status, st, sm_count);
+    return g.transB ? launch_cgemm_tc_t<false, true, TC_STAGES>(g, status, st, sm_count)
+                    : launch_cgemm_tc_t<false, false, TC_STAGES>(g, status, st, sm_count);
 }
 
 }  // namespace fc

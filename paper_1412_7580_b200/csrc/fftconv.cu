@@ -304,15 +304,21 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
             if ((small_a ? forward_small(fa, false) : forward(fa, nullptr)) != cudaSuccess) return FFTCONV_ECUDA;
             launched = true;
         }
+        // The transform of range c + 1 runs beside the contraction of range c: it is launched as
+        // that contraction's programmatic dependent, starts without waiting (it touches nothing the
+        // contraction touches) once the contraction has its operands, and completes only after it.
         for (int c = 0; c < chunks; ++c) {
             const int ky0 = (int)((long long)nc * c / chunks), ky1 = (int)((long long)nc * (c + 1) / chunks);
             g_launches.fetch_add(2, std::memory_order_relaxed);
-            if (fc::launch_r2c_small(plan->n, fb, ky0, ky1, st, launched && !big) != cudaSuccess) return FFTCONV_ECUDA;
+            const bool dep = launched && !big;
+            if (fc::launch_r2c_small(plan->n, fb, ky0, ky1, st, dep, dep) != cudaSuccess) return FFTCONV_ECUDA;
             launched = true;
             gp.ky_begin = ky0; gp.ky_count = ky1 - ky0;
             gp.overlap = big ? 0 : 1;
+            gp.shared_sms = (!big && c + 1 < chunks) ? 1 : 0;
             if (fc::launch_cgemm_tc(gp, status, st) != cudaSuccess) return FFTCONV_ECUDA;
         }
+        gp.shared_sms = 0;
         if (plan->reuse) {
             plan->cached[d.a.kind] = a_in;
             plan->cached[d.b.kind] = b_in;
