@@ -347,8 +347,8 @@ class Bench:
         fc.conv_plan_set_math(plan, math)
         if args.filter_chunks > 1:
             fc.conv_plan_set_filter_chunks(plan, args.filter_chunks)
-        if args.no_small_planes:
-            fc.conv_plan_set_small_plane_kernel(plan, False)
+        if args.small_planes != 1:
+            fc.conv_plan_set_small_plane_kernel(plan, args.small_planes)
         if tile_req:
             fc.conv_plan_set_tiling(plan, tile_req)      # -1: the plan chooses
         tile = fc.conv_plan_tile_basis(plan)
@@ -694,7 +694,7 @@ def run_ours(args):
     b = Bench(args)
     math = {"auto": fc.MATH_AUTO, "fp32": fc.MATH_FP32, "tf32": fc.MATH_TF32}[args.math]
     single = (args.config is not None or args.shape is not None or args.filter_chunks > 1
-              or args.no_small_planes)
+              or args.small_planes != 1)
     extras = not single and not args.no_extras and b.world == 1
 
     if args.fft2d or args.fft1d:
@@ -770,8 +770,8 @@ def main():
                          "roofline in the output are then those of the tiled method")
     ap.add_argument("--filter-chunks", type=int, default=1,
                     help="fprop / bprop: transform and contract the filters in this many ranges of frequency rows")
-    ap.add_argument("--no-small-planes", action="store_true",
-                    help="send the filters through the butterfly kernels instead of the small-plane kernel")
+    ap.add_argument("--small-planes", type=int, default=1, choices=[0, 1, 2],
+                    help="pruned-DFT kernels for small planes: 0 never, 1 where measured to pay (default), 2 wherever they apply")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-reuse-line", action="store_true",

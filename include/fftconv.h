@@ -148,8 +148,12 @@ int conv_accgrad(conv_plan_t* plan, const float* dy, const float* x, float* dw, 
  * operand's transform (a pass is four launches).  Likewise the inverse transform of accGrad,
  * whose result is clipped to the kh x kw filter window (Section 3.1), is a pruned inverse DFT
  * that reads whole lines for 32 adjacent planes when the window is square, at most 11 x 11 and
- * at most a quarter of the basis (n = 32 and 64).  On by default; enable == 0 sends everything
- * through the butterfly kernels (same results up to rounding). */
+ * at most a quarter of the basis (n = 32 and 64).  enable == 1 (the default) uses the forward
+ * kernel where it was measured to pay -- bases of 64 and 128; at n <= 32 planes of at most 1/16
+ * of the basis whose spectrum exceeds 96 MB; the filter operand of a chunked pass (below);
+ * otherwise the filters share the other operand's launch -- and the inverse kernel wherever it
+ * applies; enable >= 2 uses both wherever they apply; enable <= 0
+ * sends everything through the butterfly kernels.  Same results up to rounding in every mode. */
 int conv_plan_set_small_plane_kernel(conv_plan_t* plan, int enable);
 
 /* Filter spectrum through the cache (Section 6 asks for fewer passes over memory between the

@@ -250,9 +250,9 @@ def conv_plan_status(plan: Plan) -> int:
     return int(lib().conv_plan_status(plan.handle))
 
 
-def conv_plan_set_small_plane_kernel(plan: Plan, enable=True) -> None:
-    """Pruned-DFT forward kernel for operand planes of at most 13 x 13 samples (default on)."""
-    _check(lib().conv_plan_set_small_plane_kernel(plan.handle, int(bool(enable))),
+def conv_plan_set_small_plane_kernel(plan: Plan, enable=1) -> None:
+    """Pruned-DFT kernels for small planes: 0 never, 1 where measured to pay (default), 2 wherever they apply."""
+    _check(lib().conv_plan_set_small_plane_kernel(plan.handle, int(enable)),
            "conv_plan_set_small_plane_kernel")
 
 

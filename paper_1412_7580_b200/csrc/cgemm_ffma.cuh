@@ -37,7 +37,24 @@ struct GemmParams {
     // run beside this contraction; the kernel then keeps 64 KB of shared memory free (two pipeline
     // stages instead of three) and releases its dependent only after its own wait.
     int shared_sms;
+    // Both kernels: herm_n = n > 0 leaves out the bins (kx > n/2, ky in {0, n/2}) of an n x (n/2+1)
+    // half spectrum.  They are the complex conjugates of the bins (n - kx, ky) (Section 5.2: the
+    // rows ky = 0 and ky = n/2 of a real signal's spectrum are Hermitian in kx), the inverse
+    // transforms rebuild them from those, and the contraction neither reads nor writes them:
+    // n - 2 bins of n (n/2 + 1), 9.7 % at n = 16, 5.5 % at n = 32, 2.9 % at n = 64.
+    int herm_n;
 };
+
+// Bins kept by herm_n = n, and the bin of the spectra behind the b-th kept bin (kept bins in
+// increasing order: all of kx <= n/2, then ky = 1 .. n/2 - 1 of every kx > n/2).
+__host__ __device__ inline int herm_kept_bins(int n) { return n * (n / 2 + 1) - (n - 2); }
+__host__ __device__ inline int herm_bin(int b, int n) {
+    const int nc = n / 2 + 1, head = nc * nc;
+    if (b < head) return b;
+    b -= head;
+    const int kx = nc + b / (nc - 2);
+    return kx * nc + 1 + (b - (kx - nc) * (nc - 2));
+}
 
 constexpr int FG_BM = 64, FG_BN = 64, FG_BK = 16, FG_PAD = 4, FG_T = 256;
 
@@ -62,7 +79,7 @@ __global__ void __launch_bounds__(FG_T) cgemm_ffma_kernel(const GemmParams p) {
     const int tid = threadIdx.x;
     // grid: x = (row block, column block) linearised (tiled plans can have millions of row
     // blocks, more than grid.y takes), y = bin
-    const int bin = blockIdx.y;
+    const int bin = p.herm_n ? herm_bin((int)blockIdx.y, p.herm_n) : (int)blockIdx.y;
     const int n_blocks = (p.N + FG_BN - 1) / FG_BN;
     const int m_blk = (int)(blockIdx.x / n_blocks) * FG_BM, n_blk = (int)(blockIdx.x % n_blocks) * FG_BN;
     const size_t planeA = (size_t)(TA ? p.K : p.M) * p.lda,
@@ -196,7 +213,8 @@ static cudaError_t launch_cgemm_ffma_t(const GemmParams& p, dim3 grid, cudaStrea
 static cudaError_t launch_cgemm_ffma(const GemmParams& p, cudaStream_t st) {
     const long long blocks = (long long)((p.N + FG_BN - 1) / FG_BN) * ((p.M + FG_BM - 1) / FG_BM);
     if (blocks > 0x7fffffffLL || p.bins > 65535) return cudaErrorInvalidValue;
-    dim3 grid((unsigned)blocks, (unsigned)p.bins, 1);
+    if (p.herm_n && (p.herm_n < 8 || p.bins != p.herm_n * (p.herm_n / 2 + 1))) return cudaErrorInvalidValue;
+    dim3 grid((unsigned)blocks, (unsigned)(p.herm_n ? herm_kept_bins(p.herm_n) : p.bins), 1);
     if (p.transA) return p.transB ? launch_cgemm_ffma_t<true, true>(p, grid, st) : launch_cgemm_ffma_t<true, false>(p, grid, st);
     return p.transB ? launch_cgemm_ffma_t<false, true>(p, grid, st) : launch_cgemm_ffma_t<false, false>(p, grid, st);
 }

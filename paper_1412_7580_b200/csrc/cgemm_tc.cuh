@@ -66,6 +66,7 @@ struct TcParams {
     int bins_run;               // bins contracted by this launch (all of them, or a ky range of every kx)
     int nc, ky_begin, ky_count; // ky_count > 0: local bin b -> kx = b / ky_count, ky = ky_begin + b % ky_count
     int late_trigger;           // let the dependent launch start after this one's wait instead of before it
+    int herm_n;                 // > 0: the launch runs the kept bins of GemmParams::herm_n (local bin -> herm_bin)
 };
 
 static inline bool tc_shape_supported(int M, int N, int K) {
@@ -240,6 +241,7 @@ cgemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     const int num_tiles = p.bins_run * p.m_tiles * p.n_tiles;
     // local bin of this launch -> bin of the spectra
     auto global_bin = [&](int b) {
+        if (p.herm_n) return herm_bin(b, p.herm_n);
         if (p.ky_count == 0) return b;
         const int kx = b / p.ky_count;
         return kx * p.nc + p.ky_begin + (b - kx * p.ky_count);
@@ -449,6 +451,12 @@ static cudaError_t launch_cgemm_tc_t(const GemmParams& g, int* status, cudaStrea
     p.wait_cycles = g.wait_cycles > 0 ? g.wait_cycles : TC_WAIT_CYCLES;
     p.bins_run = g.bins; p.nc = g.nc; p.ky_begin = g.ky_begin; p.ky_count = 0;
     p.late_trigger = g.shared_sms ? 1 : 0;
+    p.herm_n = 0;
+    if (g.herm_n) {
+        if (g.ky_count > 0 || g.herm_n < 8 || g.bins != g.herm_n * (g.herm_n / 2 + 1)) return cudaErrorInvalidValue;
+        p.herm_n = g.herm_n;
+        p.bins_run = herm_kept_bins(g.herm_n);
+    }
     if (g.ky_count > 0) {
         if (g.nc < 1 || g.bins % g.nc != 0 || g.ky_begin < 0 || g.ky_begin + g.ky_count > g.nc)
             return cudaErrorInvalidValue;

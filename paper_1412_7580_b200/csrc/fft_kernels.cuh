@@ -821,12 +821,20 @@ c2r_kernel(const __grid_constant__ CUtensorMap tmS, const FftParams p) {
             // that the two warps holding the packed rows do no more work than the others.
             constexpr bool WIDE_COMBINE = (N <= 64);
             if constexpr (WIDE_COMBINE) {
-                for (int it = tid; it < G * N; it += T) {
+                // The two rows are Hermitian in kx, and their bins kx > N/2 are never read: the
+                // thread of kx <= N/2 also forms Z[N - kx] = conj X_0[kx] + i conj X_{N/2}[kx]
+                // (the contraction leaves those bins out, see GemmParams::herm_n).
+                for (int it = tid; it < G * (M + 1); it += T) {
                     const int g = it % G, kx = it / G;
                     float* a = sStage + (size_t)kx * NC * G + g;
                     const float x0r = a[0], x0i = a[B * G], xnr = a[M * G], xni = a[(B + M) * G];
                     a[0] = x0r - xni;
                     a[B * G] = x0i + xnr;
+                    if (kx > 0 && kx < M) {
+                        float* m = sStage + (size_t)(N - kx) * NC * G + g;
+                        m[0] = x0r + xni;
+                        m[B * G] = xnr - x0i;
+                    }
                 }
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before the next TMA fill
                 __syncthreads();

@@ -285,7 +285,8 @@ constexpr int SMALLINV_WARPS = 4;
 
 template <int N, int K>
 __global__ void __launch_bounds__(SMALLINV_WARPS * 32)
-c2r_small_kernel(const __grid_constant__ CUtensorMap tmS, const SmallInvParams p) {
+c2r_small_kernel(const __grid_constant__ CUtensorMap tmS, const __grid_constant__ CUtensorMap tmH,
+                 const SmallInvParams p) {
     constexpr int NC = N / 2 + 1, NQ = N / 4, TWS = 128 / N, MASK = N - 1, NST = SmallInvCfg<N>::NST;
     constexpr int ROW_FLOATS = 2 * N * 32;              // one frequency row: [part*N + kx][32 planes]
     constexpr int KSQ = K * K;
@@ -325,9 +326,17 @@ c2r_small_kernel(const __grid_constant__ CUtensorMap tmS, const SmallInvParams p
     auto issue = [&]() {
         if (lane == 0) {
             const int cb = (int)(iss_blk % p.cblocks), r = (int)(iss_blk / p.cblocks);
-            fk_mbar_expect_tx(bars + 8u * iss_stage, (uint32_t)(ROW_FLOATS * 4));
-            fk_tma_load_4d(fk_smem_u32(ring + (size_t)iss_stage * ROW_FLOATS), &tmS, cb * 32, r,
-                           member + split * iss_row, 0, bars + 8u * iss_stage);
+            const int ky = member + split * iss_row;
+            const uint32_t dst = fk_smem_u32(ring + (size_t)iss_stage * ROW_FLOATS);
+            if (ky == 0 || ky == N / 2) {
+                // Hermitian rows: only the lines kx <= N/2 of either part are fetched
+                fk_mbar_expect_tx(bars + 8u * iss_stage, (uint32_t)(2 * (N / 2 + 1) * 32 * 4));
+                fk_tma_load_4d(dst, &tmH, cb * 32, r, ky, 0, bars + 8u * iss_stage);
+                fk_tma_load_4d(dst + (uint32_t)(N * 32 * 4), &tmH, cb * 32, r, ky, N, bars + 8u * iss_stage);
+            } else {
+                fk_mbar_expect_tx(bars + 8u * iss_stage, (uint32_t)(ROW_FLOATS * 4));
+                fk_tma_load_4d(dst, &tmS, cb * 32, r, ky, 0, bars + 8u * iss_stage);
+            }
         }
         if (++iss_row == my_rows) { iss_row = 0; iss_blk += stride; }
         if (++iss_stage == NST) iss_stage = 0;
@@ -350,6 +359,19 @@ c2r_small_kernel(const __grid_constant__ CUtensorMap tmS, const SmallInvParams p
         if (ok && !fk_wait_or_report(bars + 8u * s, (phase >> s) & 1u, p.wait_cycles, p.status)) ok = false;
         phase ^= (1u << s);
         if (ok) {
+            if (ky == 0 || ky == N / 2) {
+                // These two rows are Hermitian in kx and their bins kx > N/2 are never read (the
+                // contraction leaves them out, see GemmParams::herm_n): every lane rebuilds them
+                // in its own column of the row.
+                float* wr = ring + (size_t)s * ROW_FLOATS + lane;
+                float* wi = wr + N * 32;
+#pragma unroll
+                for (int kx = N / 2 + 1; kx < N; ++kx) {
+                    wr[kx * 32] = wr[(N - kx) * 32];
+                    wi[kx * 32] = -wi[(N - kx) * 32];
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // before the next TMA fill of this stage
+            }
             const float* xr = ring + (size_t)s * ROW_FLOATS + lane;     // [kx][32]
             const float* xi = xr + N * 32;
             float Zr[K], Zi[K];
@@ -443,15 +465,16 @@ static inline bool small_inv_supported(int n, int hc, int wc) {
     return hc <= 5 || hc == 7 || hc == 9 || hc == 11;
 }
 
+// box_kx: lines of one box (2 N: a whole row, both parts; N/2 + 1: the kept half of one part)
 template <int N>
-static bool small_inv_map(CUtensorMap* map, const float* spec, const FftParams& p) {
+static bool small_inv_map(CUtensorMap* map, const float* spec, const FftParams& p, int box_kx) {
     tc_encode_fn enc = tc_get_encode();
     if (!enc) return false;
     constexpr int NC = N / 2 + 1;
     const cuuint64_t mat = (cuuint64_t)p.R * p.ld * 4;
     cuuint64_t dims[4] = {(cuuint64_t)p.C, (cuuint64_t)p.R, (cuuint64_t)NC, (cuuint64_t)2 * N};
     cuuint64_t strides[3] = {(cuuint64_t)p.ld * 4, mat, mat * NC};
-    cuuint32_t box[4] = {32u, 1u, 1u, (cuuint32_t)2 * N};
+    cuuint32_t box[4] = {32u, 1u, 1u, (cuuint32_t)box_kx};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<float*>(spec), dims, strides, box,
                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
@@ -463,9 +486,11 @@ static cudaError_t launch_c2r_small_nk(const FftParams& f, cudaStream_t st) {
     if constexpr (2 * K > N) {
         return cudaErrorNotSupported;
     } else {
-        CUtensorMap tm;
+        CUtensorMap tm, tmh;
         memset(&tm, 0, sizeof(tm));
-        if (!small_inv_map<N>(&tm, f.spec_in, f)) return cudaErrorInvalidValue;
+        memset(&tmh, 0, sizeof(tmh));
+        if (!small_inv_map<N>(&tm, f.spec_in, f, 2 * N) || !small_inv_map<N>(&tmh, f.spec_in, f, N / 2 + 1))
+            return cudaErrorInvalidValue;
         SmallInvParams p{};
         p.real_out = f.real_out; p.n = N; p.k = K; p.R = f.R; p.C = f.C;
         p.cblocks = (f.C + 31) / 32;
@@ -481,7 +506,7 @@ static cudaError_t launch_c2r_small_nk(const FftParams& f, cudaStream_t st) {
         int grid = 0;
         cudaError_t e = persistent_grid(reinterpret_cast<const void*>(kern), SMALLINV_WARPS * 32, smem, ctas, &grid);
         if (e != cudaSuccess) return e;
-        return dep_launch(f.overlap != 0, kern, dim3(grid), dim3(SMALLINV_WARPS * 32), smem, st, tm, p);
+        return dep_launch(f.overlap != 0, kern, dim3(grid), dim3(SMALLINV_WARPS * 32), smem, st, tm, tmh, p);
     }
 }
 template <int N>

@@ -71,7 +71,7 @@ struct conv_plan_s {
     cudaEvent_t ev[5];
     bool ev_made;
     long long wait_cycles;  // limit of a bounded device-side wait in SM cycles; 0 = the kernels' default
-    int small_planes;       // small operand planes (filters) take the pruned-DFT forward kernel
+    int small_planes;       // pruned-DFT kernels for small planes: 0 never, 1 where measured to pay, 2 wherever they apply
     int filter_chunks;      // > 1: the filter spectrum is produced and contracted in this many bin ranges
 };
 
@@ -265,8 +265,20 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     // Small planes (the filters of fprop and bprop) take the pruned-DFT kernel, whose stores are
     // whole 128-byte lines; it runs after the other operand's transform, as its programmatic
     // dependent where that transform is a one-pass kernel.
-    auto is_small = [&](const fc::FftParams& f) {
-        return plan->small_planes && !f.win && fc::small_supported(plan->n, f.h, f.w);
+    // Mode 1 (default) takes it where it was measured to pay: at n >= 64 (passes 1.1-1.4 x
+    // shorter); at n <= 32 only for planes of at most 1/16 of the basis whose spectrum is much
+    // larger than the L2 (mid and deep layers: 1-2 % shorter passes), because otherwise the one
+    // launch for both operands is as fast or faster (the filter spectrum is bound by the store
+    // rate either way, a fourth launch costs 3-5 us on small layers, and wider filters at
+    // n <= 32 are 7-25 % slower as direct sums); and for the filter operand of a chunked pass.
+    // Mode 2 takes it wherever it applies.
+    const bool tensor = resolve_math(*plan, d) == FFTCONV_MATH_TF32;
+    const bool want_chunks = plan->filter_chunks > 1 && tensor && !timing;
+    auto is_small = [&](const fc::FftParams& f, bool filter_operand) {
+        if (!plan->small_planes || f.win || !fc::small_supported(plan->n, f.h, f.w)) return false;
+        if (plan->small_planes == 2 || plan->n >= 64 || (filter_operand && want_chunks)) return true;
+        const double spec_bytes = 8.0 * plan->bins * (double)f.R * f.ld;
+        return 16 * f.h * f.w <= plan->n * plan->n && spec_bytes >= 96e6;
     };
     // dep: another forward transform of this pass was launched just before; the small-plane kernel
     // then runs beside it (neither touches the other's data) and completes only after it.
@@ -277,8 +289,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     };
     mark(0);
     const fc::FftParams fa = operand(d.a, a_in, specA), fb = operand(d.b, b_in, specB);
-    const bool small_a = need_a && is_small(fa), small_b = need_b && is_small(fb);
-    const bool tensor = resolve_math(*plan, d) == FFTCONV_MATH_TF32;
+    const bool small_a = need_a && is_small(fa, false), small_b = need_b && is_small(fb, true);
     // the kernels of a pass overlap their ramp-up with the predecessor's drain where that
     // was measured to pay (see dep_launch.cuh)
     const bool overlap = !big && !timing && (tensor || plan->n >= 32 || d.K <= 64);
@@ -290,10 +301,12 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     gp.transA = d.transA; gp.transB = d.transB; gp.conjA = d.conjA; gp.conjB = d.conjB;
     gp.wait_cycles = plan->wait_cycles;
     gp.nc = plan->n / 2 + 1;
+    // one-pass inverse transforms (n <= 64) rebuild the conjugate bins of the rows ky = 0 and
+    // ky = n/2 themselves, so the contraction leaves them out
+    const int herm_n = (!big && plan->n <= 64) ? plan->n : 0;
 
     const int nc = plan->n / 2 + 1;
-    const int chunks = (plan->filter_chunks > 1 && small_b && tensor && !timing)
-                           ? (plan->filter_chunks < nc ? plan->filter_chunks : nc) : 1;
+    const int chunks = (want_chunks && small_b) ? (plan->filter_chunks < nc ? plan->filter_chunks : nc) : 1;
     if (chunks > 1) {
         // Filter spectrum through the L2: the small-plane kernel can produce any range of rows
         // ky, so the filter operand is transformed and contracted range by range -- each part
@@ -344,6 +357,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     gp.overlap = (overlap && (need_a || need_b)) ? 1 : 0;       // predecessor: this pass's forward transforms
+    gp.herm_n = herm_n;
     cudaError_t ge;
     if (tensor) ge = fc::launch_cgemm_tc(gp, status, st);
     else ge = fc::launch_cgemm_ffma(gp, st);
@@ -654,7 +668,7 @@ FFTCONV_API int conv_plan_set_filter_chunks(conv_plan_t* plan, int chunks) {
 
 FFTCONV_API int conv_plan_set_small_plane_kernel(conv_plan_t* plan, int enable) {
     if (!plan) return FFTCONV_EINVAL;
-    plan->small_planes = enable ? 1 : 0;
+    plan->small_planes = enable <= 0 ? 0 : (enable >= 2 ? 2 : 1);
     return FFTCONV_OK;
 }
 

@@ -13,8 +13,9 @@ def relerr(got, ref):
     return float(np.max(np.abs(got - ref)) / np.max(np.abs(ref)))
 
 
+@pytest.mark.parametrize("small", [1, 2])
 @pytest.mark.parametrize("dims", [(16, 24, 40, 13, 13, 3, 3, 16), (3, 5, 7, 27, 30, 5, 4, 32)])
-def test_reuse_matches_plain_passes_and_oracle(dims):
+def test_reuse_matches_plain_passes_and_oracle(dims, small):
     import torch
     import oracle
     import paper_1412_7580_b200 as fc
@@ -29,22 +30,25 @@ def test_reuse_matches_plain_passes_and_oracle(dims):
                 torch.full((s.fp, s.f, s.kh, s.kw), float("nan"), device="cuda"))
 
     plain = fc.conv_plan(*s.args())
+    fc.conv_plan_set_small_plane_kernel(plain, small)
     fc.conv_plan_alloc_workspace(plain)
     y0, dx0, dw0 = outputs()
     fc.conv_fprop(plain, xd, wd, y0); fc.conv_bprop(plain, dyd, wd, dx0); fc.conv_accgrad(plain, dyd, xd, dw0)
 
     p = fc.conv_plan(*s.args())
-    small = fc.conv_plan_workspace_bytes(p)
+    fc.conv_plan_set_small_plane_kernel(p, small)
+    plain_bytes = fc.conv_plan_workspace_bytes(p)
     fc.conv_plan_set_spectrum_reuse(p, True)
-    assert fc.conv_plan_workspace_bytes(p) >= small
+    assert fc.conv_plan_workspace_bytes(p) >= plain_bytes
     ws = fc.conv_plan_alloc_workspace(p)
     ws.view(torch.float32)[64:].fill_(float("nan"))
     y1, dx1, dw1 = outputs()
     before = fc.fftconv_launch_count()
     fc.conv_fprop(p, xd, wd, y1); fc.conv_bprop(p, dyd, wd, dx1); fc.conv_accgrad(p, dyd, xd, dw1)
-    # fprop: x, w (small planes: a launch of its own), contraction, inverse; bprop: dy only;
-    # accGrad: no forward transform at all -- three forward transforms saved
-    assert fc.fftconv_launch_count() - before == 4 + 3 + 2
+    # fprop: x and w (one launch at these bases; with the small-plane kernel forced, w has a
+    # launch of its own), contraction, inverse; bprop: dy only; accGrad: no forward transform
+    # at all -- three forward transforms saved
+    assert fc.fftconv_launch_count() - before == (4 if small == 2 else 3) + 3 + 2
     torch.cuda.synchronize()
     for a, b in ((y0, y1), (dx0, dx1), (dw0, dw1)):
         assert torch.equal(a, b)                                  # same kernels, same spectra

@@ -77,7 +77,7 @@ def test_small_plane_kernel_on_off_and_chunked(dims, math):
     x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
     ref_y, ref_dx = oracle.fprop(x, w), oracle.bprop(dy, w, s.h, s.w)
     ref_dw = oracle.accgrad(dy, x, s.kh, s.kw)
-    for small, chunks in ((1, 1), (0, 1), (1, 3), (1, 100)):
+    for small, chunks in ((2, 1), (1, 1), (0, 1), (1, 3), (2, 100)):
         y, dx, dw, dw2, eff = run(s, x, w, dy, math, small, chunks)
         assert np.all(np.isfinite(y)) and np.all(np.isfinite(dx)) and np.all(np.isfinite(dw)), (small, chunks)
         assert relerr(y, ref_y) <= TOL[eff[0]], (small, chunks)
