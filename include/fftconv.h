@@ -240,8 +240,10 @@ int conv_plan_enable_stage_timing(conv_plan_t* plan, int enable);
 
 /* Waits for the last pass issued with timing enabled and writes durations in
  * milliseconds to out_ms[0..3]: forward FFT of the first operand (mode 1: of both
- * operands, the one fused kernel), forward FFT of the second operand (mode 1:
- * zero), contraction, inverse FFT.  EINVAL if timing is off or no pass has run. */
+ * operands where they share one kernel), forward FFT of the second operand
+ * (exactly zero where it had no launch of its own: mode 1 unless the operand takes
+ * the small-plane kernel), contraction, inverse FFT.  EINVAL if timing is off or no
+ * pass has run. */
 int conv_plan_stage_times_ms(conv_plan_t* plan, float* out_ms);
 
 /* Bare batched 2-D real-to-complex transform (Supplement 8.2 definition,

@@ -68,6 +68,7 @@ struct conv_plan_s {
     const float* cached[3]; // reuse: tensor whose spectrum sits in region 0 (x), 1 (w), 2 (dy)
     int timing;             // record events around the four kernels of a pass
     bool timed;             // a timed pass has been issued
+    bool second_stage_used; // the timed pass launched something between the second and third event
     cudaEvent_t ev[5];
     bool ev_made;
     long long wait_cycles;  // limit of a bounded device-side wait in SM cycles; 0 = the kernels' default
@@ -341,6 +342,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         // both forward transforms in one launch: one ramp-up, one tail
         if (forward(fa, &fb) != cudaSuccess) return FFTCONV_ECUDA;
         mark(1);
+        if (timing) plan->second_stage_used = false;
     } else {
         // one kernel per operand (small planes, spectrum reuse, or timing mode 2)
         bool launched = false;
@@ -349,6 +351,7 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
         mark(1);
         if (need_b && !small_b) { if (forward(fb, nullptr) != cudaSuccess) return FFTCONV_ECUDA; launched = true; }
         if (need_b && small_b) { if (forward_small(fb, launched) != cudaSuccess) return FFTCONV_ECUDA; }
+        if (timing) plan->second_stage_used = need_b;
     }
     mark(2);
     if (plan->reuse) {
@@ -700,6 +703,7 @@ FFTCONV_API int conv_plan_stage_times_ms(conv_plan_t* plan, float* out_ms) {
     for (int i = 0; i < 4; ++i)
         if (cudaEventElapsedTime(&out_ms[i], plan->ev[i], plan->ev[i + 1]) != cudaSuccess)
             return FFTCONV_ECUDA;
+    if (!plan->second_stage_used) out_ms[1] = 0.0f;      // nothing was launched there: two adjacent events
     return FFTCONV_OK;
 }
 
