@@ -601,11 +601,19 @@ class Bench:
             p = fc.conv_plan(*s.args())
             if tile == "auto":
                 fc.conv_plan_set_tiling(p, fc.TILE_AUTO)
-            ws = fc.conv_plan_alloc_workspace(p)
             xd, wd, dyd = (torch.from_numpy(a).cuda() for a in (x, w, dy))
             y = torch.full((s.S, s.fp, s.oh, s.ow), float("nan"), device="cuda")
             dx = torch.full((s.S, s.f, s.h, s.w), float("nan"), device="cuda")
             dw = torch.full((s.fp, s.f, s.kh, s.kw), float("nan"), device="cuda")
+            tuned = None
+            if tile == "tuned":
+                # measured choice: the library times a step for every admissible basis
+                # (candidates that need more than 16 GB of workspace are left out by the library)
+                nbytes = max(fc.conv_plan_workspace_bytes(p), min(fc.conv_plan_tune_workspace_bytes(p), 16 << 30))
+                ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+                _, tuned = fc.conv_plan_tune_tiling(p, xd, wd, dyd, y, dx, dw, ws, reps=2)
+            else:
+                ws = fc.conv_plan_alloc_workspace(p)
             calls = [lambda: fc.conv_fprop(p, xd, wd, y), lambda: fc.conv_bprop(p, dyd, wd, dx),
                      lambda: fc.conv_accgrad(p, dyd, xd, dw)]
             ms = []
@@ -624,6 +632,8 @@ class Bench:
                    "math": ["tf32" if fc.conv_plan_pass_math(p, k) == fc.MATH_TF32 else "f32" for k in range(3)],
                    "finite_and_status_ok": ok, "ms": ms, "roofline_frac": fr,
                    "gflops_equiv": [2.0 * s.macs / (m * 1e-3) / 1e9 for m in ms]}
+            if tuned is not None:
+                rec["tuner_step_ms"] = {str(k): v for k, v in tuned.items()}
             recs.append(rec)
             if fh:
                 fh.write(json.dumps(rec) + "\n"); fh.flush()
@@ -785,7 +795,8 @@ def main():
     ap.add_argument("--sweep-only", action="store_true", help="run the seeded sweep points only (timing)")
     ap.add_argument("--sweep-points", type=int, default=1000)
     ap.add_argument("--sweep-out", default=None, help="JSON lines, one per sweep point")
-    ap.add_argument("--sweep-tile", default="off", choices=["off", "auto"])
+    ap.add_argument("--sweep-tile", default="off", choices=["off", "auto", "tuned"],
+                    help="tile basis of the sweep points: untiled, the plan's byte model, or measured")
     ap.add_argument("--fft2d", action="store_true", help="throughput table of the bare 2-D transforms")
     ap.add_argument("--fft1d", action="store_true", help="throughput table of the bare 1-D transforms")
     ap.add_argument("--mb", type=int, default=256, help="megabytes of samples per launch for --fft2d / --fft1d")

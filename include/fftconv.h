@@ -205,6 +205,29 @@ int conv_plan_invalidate_spectra(conv_plan_t* plan);
 #define FFTCONV_TILE_AUTO (-1)
 int conv_plan_set_tiling(conv_plan_t* plan, int n_tile);
 
+/* Measured choice of the tile basis (Section 3.4: the paper's autotuner times the candidate
+ * bases of a problem size and keeps the fastest; FFTCONV_TILE_AUTO above ranks them with a byte
+ * model instead).  Runs one warm-up and `reps` (1..100) timed training steps -- fprop, bprop,
+ * accGrad -- for the untiled basis (where the plan's n <= 128) and for every admissible tile
+ * basis in {8, 16, 32, 64} below n, on the caller's tensors (device pointers, the layouts of
+ * conv_fprop / conv_bprop / conv_accgrad), timed with CUDA events on `cuda_stream`, and leaves
+ * the plan on the fastest basis with `workspace` lent to it.  y, dx and dw are overwritten (the
+ * last candidate's results, which equal every other candidate's up to rounding).  `workspace`:
+ * device memory, 256-byte aligned; conv_plan_tune_workspace_bytes(plan) is the largest workspace
+ * of any candidate, and a candidate that needs more than `workspace_bytes` is left out (small
+ * tile bases of large planes can need many times the untiled workspace); it stays with the
+ * caller and is the plan's workspace afterwards.  *chosen_basis (host, may be null) receives the basis, 0 = untiled; step_ms (host,
+ * may be null) receives FFTCONV_TUNE_CANDIDATES step times in milliseconds in the order
+ * untiled, 8, 16, 32, 64, negative where a candidate is not admissible or was left out.
+ * Synchronises the stream.  EUNSUPPORTED with spectrum reuse enabled or when no candidate is
+ * admissible and fits the workspace; ECUDA when a run fails or a device wait gives up (the plan
+ * then keeps the basis it had). */
+#define FFTCONV_TUNE_CANDIDATES 5
+size_t conv_plan_tune_workspace_bytes(conv_plan_t* plan);
+int conv_plan_tune_tiling(conv_plan_t* plan, const float* x, const float* w, const float* dy,
+                          float* y, float* dx, float* dw, void* workspace, size_t workspace_bytes,
+                          int reps, void* cuda_stream, int* chosen_basis, float* step_ms);
+
 /* The tile basis in use, 0 when tiling is off. */
 int conv_plan_tile_basis(const conv_plan_t* plan);
 

@@ -21,7 +21,7 @@ EXPORTS = (
     "conv_plan", "conv_plan_set_math", "conv_plan_effective_math", "conv_plan_pass_math",
     "conv_plan_workspace_bytes",
     "conv_plan_set_workspace", "conv_plan_set_spectrum_reuse", "conv_plan_invalidate_spectra",
-    "conv_plan_set_tiling", "conv_plan_tile_basis",
+    "conv_plan_set_tiling", "conv_plan_tile_basis", "conv_plan_tune_tiling", "conv_plan_tune_workspace_bytes",
     "conv_fprop", "conv_fprop_noalloc", "conv_bprop", "conv_accgrad", "conv_plan_status",
     "conv_plan_set_wait_limit", "conv_plan_set_small_plane_kernel", "conv_plan_set_filter_chunks",
     "conv_plan_destroy", "conv_plan_enable_stage_timing", "conv_plan_stage_times_ms", "fft2d_r2c", "fft2d_c2r", "fft1d_r2c", "fft1d_c2r", "fftconv_bin_contract",
@@ -58,6 +58,10 @@ def lib():
         L.conv_plan_invalidate_spectra.argtypes = [p]
         L.conv_plan_set_tiling.argtypes = [p, i]
         L.conv_plan_tile_basis.argtypes = [p]
+        L.conv_plan_tune_workspace_bytes.argtypes = [p]
+        L.conv_plan_tune_workspace_bytes.restype = z
+        L.conv_plan_tune_tiling.argtypes = [p, p, p, p, p, p, p, p, z, i, p, ctypes.POINTER(i),
+                                            ctypes.POINTER(fl)]
         L.conv_fprop.argtypes = [p, p, p, p, p]
         L.conv_fprop_noalloc.argtypes = [p, p, p, p, p]
         L.conv_bprop.argtypes = [p, p, p, p, p]
@@ -80,8 +84,8 @@ def lib():
         L.fftconv_launch_count.restype = ctypes.c_ulonglong
         for name in EXPORTS:
             fn = getattr(L, name)
-            if name not in ("conv_plan_workspace_bytes", "fftconv_status_string",
-                            "fftconv_launch_count"):
+            if name not in ("conv_plan_workspace_bytes", "conv_plan_tune_workspace_bytes",
+                            "fftconv_status_string", "fftconv_launch_count"):
                 fn.restype = i
         _lib = L
     return _lib
@@ -192,6 +196,36 @@ def conv_plan_set_tiling(plan: Plan, n_tile: int) -> None:
 
 def conv_plan_tile_basis(plan: Plan) -> int:
     return lib().conv_plan_tile_basis(plan.handle)
+
+
+TUNE_CANDIDATES = (0, 8, 16, 32, 64)
+
+
+def conv_plan_tune_workspace_bytes(plan: Plan) -> int:
+    """Bytes of the largest workspace any candidate basis of conv_plan_tune_tiling needs."""
+    return int(lib().conv_plan_tune_workspace_bytes(plan.handle))
+
+
+def conv_plan_tune_tiling(plan: Plan, x, w, dy, y, dx, dw, workspace, reps=3, stream=None):
+    """Measured choice of the tile basis: times a training step for the untiled basis and every
+    admissible tile basis on the given CUDA tensors and leaves the plan on the fastest, with
+    `workspace` lent to it (a CUDA tensor; conv_plan_tune_workspace_bytes(plan) bytes hold every
+    candidate, a candidate that needs more than the tensor has is left out).  Returns (chosen basis, {basis: step time in ms}) with 0 for the untiled basis."""
+    nbytes = workspace.numel() * workspace.element_size()
+    chosen = ctypes.c_int(-1)
+    ms = (ctypes.c_float * len(TUNE_CANDIDATES))()
+    _check(lib().conv_plan_tune_tiling(plan.handle,
+                                       _dev(x, (plan.S, plan.f, plan.h, plan.w), "x"),
+                                       _dev(w, (plan.fp, plan.f, plan.kh, plan.kw), "w"),
+                                       _dev(dy, (plan.S, plan.fp, plan.oh, plan.ow), "dy"),
+                                       _dev(y, (plan.S, plan.fp, plan.oh, plan.ow), "y"),
+                                       _dev(dx, (plan.S, plan.f, plan.h, plan.w), "dx"),
+                                       _dev(dw, (plan.fp, plan.f, plan.kh, plan.kw), "dw"),
+                                       ctypes.c_void_p(workspace.data_ptr()), nbytes, int(reps),
+                                       _stream_ptr(stream), ctypes.byref(chosen), ms),
+           "conv_plan_tune_tiling")
+    plan.workspace = workspace
+    return int(chosen.value), {b: float(ms[i]) for i, b in enumerate(TUNE_CANDIDATES) if ms[i] >= 0.0}
 
 
 def conv_plan_invalidate_spectra(plan: Plan) -> None:

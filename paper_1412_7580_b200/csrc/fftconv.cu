@@ -544,6 +544,81 @@ FFTCONV_API int conv_plan_set_tiling(conv_plan_t* plan, int n_tile) {
     return FFTCONV_OK;
 }
 
+// ---------------------------------------------------------------------------
+// Measured choice of the tile basis (the paper's autotuner, Section 3.4, times the candidate
+// bases of a problem and keeps the fastest).
+// ---------------------------------------------------------------------------
+namespace {
+const int kTuneCand[FFTCONV_TUNE_CANDIDATES] = {0, 8, 16, 32, 64};      // 0: untiled
+}
+
+FFTCONV_API size_t conv_plan_tune_workspace_bytes(conv_plan_t* plan) {
+    if (!plan || plan->reuse) return 0;
+    const int keep = plan->n != plan->n_full ? plan->n : 0;
+    size_t m = 0;
+    for (int i = 0; i < FFTCONV_TUNE_CANDIDATES; ++i) {
+        if (kTuneCand[i] >= plan->n_full && kTuneCand[i] != 0) continue;
+        if (conv_plan_set_tiling(plan, kTuneCand[i]) != FFTCONV_OK) continue;
+        const size_t b = conv_plan_workspace_bytes(plan);
+        if (b > m) m = b;
+    }
+    if (conv_plan_set_tiling(plan, keep) != FFTCONV_OK) return 0;
+    return m;
+}
+
+FFTCONV_API int conv_plan_tune_tiling(conv_plan_t* plan, const float* x, const float* w, const float* dy,
+                                      float* y, float* dx, float* dw, void* workspace,
+                                      size_t workspace_bytes, int reps, void* cuda_stream,
+                                      int* chosen_basis, float* step_ms) {
+    if (!plan || !x || !w || !dy || !y || !dx || !dw || !workspace) return FFTCONV_EINVAL;
+    if (plan->reuse) return FFTCONV_EUNSUPPORTED;
+    if (reps < 1) reps = 1;
+    if (reps > 100) reps = 100;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    const int keep = plan->n != plan->n_full ? plan->n : 0;
+    const int timing_keep = plan->timing;
+    plan->timing = 0;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        if (e0) cudaEventDestroy(e0);
+        plan->timing = timing_keep;
+        return FFTCONV_ECUDA;
+    }
+    int best = -1, rc = FFTCONV_OK;
+    float best_ms = 0.0f;
+    for (int i = 0; i < FFTCONV_TUNE_CANDIDATES; ++i) {
+        if (step_ms) step_ms[i] = -1.0f;
+        const int cand = kTuneCand[i];
+        if (cand != 0 && cand >= plan->n_full) continue;
+        if (conv_plan_set_tiling(plan, cand) != FFTCONV_OK) continue;                  // not admissible
+        if (conv_plan_set_workspace(plan, workspace, workspace_bytes) != FFTCONV_OK) continue;
+        bool ok = true;
+        for (int r = -1; r < reps && ok; ++r) {                                       // r = -1: warm-up
+            if (r == 0) ok = cudaEventRecord(e0, st) == cudaSuccess;
+            ok = ok && run_pass(plan, PASS_FPROP, x, w, y, 0, st) == FFTCONV_OK
+                    && run_pass(plan, PASS_BPROP, dy, w, dx, 0, st) == FFTCONV_OK
+                    && run_pass(plan, PASS_ACCGRAD, dy, x, dw, 0, st) == FFTCONV_OK;
+        }
+        float ms = 0.0f;
+        ok = ok && cudaEventRecord(e1, st) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess
+                && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess && conv_plan_status(plan) == FFTCONV_OK;
+        if (!ok) { rc = FFTCONV_ECUDA; break; }
+        ms /= (float)reps;
+        if (step_ms) step_ms[i] = ms;
+        if (best < 0 || ms < best_ms) { best = cand; best_ms = ms; }
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    plan->timing = timing_keep;
+    if (rc == FFTCONV_OK && best < 0) rc = FFTCONV_EUNSUPPORTED;
+    // leave the plan on the fastest basis (on the one it had, after a failure) with the caller's workspace
+    if (conv_plan_set_tiling(plan, rc == FFTCONV_OK ? best : keep) != FFTCONV_OK ||
+        conv_plan_set_workspace(plan, workspace, workspace_bytes) != FFTCONV_OK)
+        return rc == FFTCONV_OK ? FFTCONV_EWORKSPACE : rc;
+    if (rc == FFTCONV_OK && chosen_basis) *chosen_basis = best;
+    return rc;
+}
+
 FFTCONV_API int conv_plan_tile_basis(const conv_plan_t* plan) {
     if (!plan) return FFTCONV_EINVAL;
     return plan->n != plan->n_full ? plan->n : 0;

@@ -67,6 +67,12 @@ def test_plan_validation(L):
     assert L.conv_plan_tile_basis(h) in (8, 16, 32, 64)
     assert L.conv_plan_set_tiling(h, 0) == b.EUNSUPPORTED
     assert L.conv_plan_set_tiling(h, b.TILE_AUTO) == b.OK and L.conv_plan_tile_basis(h) > 0
+    # the measured tuner: workspace of the largest candidate, plan left on the basis it had;
+    # null tensors are refused before anything runs
+    basis = L.conv_plan_tile_basis(h)
+    assert L.conv_plan_tune_workspace_bytes(h) >= L.conv_plan_workspace_bytes(h)
+    assert L.conv_plan_tile_basis(h) == basis
+    assert L.conv_plan_tune_tiling(h, None, None, None, None, None, None, None, 0, 1, None, None, None) == b.EINVAL
     assert L.conv_plan_destroy(h) == b.OK
     assert plan(8, 4, 8, 4, 4, 3, 3, 4) == b.EUNSUPPORTED
     # rectangular planes and kernels are accepted

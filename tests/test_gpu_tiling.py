@@ -163,3 +163,49 @@ def test_tiled_layers_at_benchmark_scale_sampled(dims, n_tile):
     a = float(np.sum(y * dy)); b = float(np.sum(dx * x)); c = float(np.sum(dw * w))
     scale = np.sqrt(float(np.sum(y * y)) * float(np.sum(dy.astype(np.float64) ** 2)))
     assert abs(a - b) <= 10 * tol * scale and abs(a - c) <= 10 * tol * scale
+
+
+@pytest.mark.parametrize("dims", [(2, 24, 40, 64, 64, 3, 3, 64), (3, 5, 7, 31, 31, 5, 5, 32),
+                                  (1, 6, 4, 150, 140, 5, 3, 256)])
+def test_measured_choice_of_the_tile_basis(dims):
+    """conv_plan_tune_tiling (Section 3.4: the autotuner times the candidate bases): every
+    admissible basis is timed, the plan ends on the fastest with the lent workspace, and the
+    results of the tuning run and of a pass after it match the oracle."""
+    import torch
+    import oracle
+    import paper_1412_7580_b200 as fc
+    from paper_1412_7580_b200 import workloads as wl
+    s = wl.ConvShape("tune", *dims, cfg=13, point=sum(dims))
+    x, w, dy = wl.make_x(s), wl.make_w(s), wl.make_dy(s)
+    xd, wd, dyd = (torch.from_numpy(a).cuda() for a in (x, w, dy))
+    p = fc.conv_plan(*s.args())
+    need = fc.conv_plan_tune_workspace_bytes(p)
+    assert need >= fc.conv_plan_workspace_bytes(p)
+    ws = torch.empty(need + 512, dtype=torch.uint8, device="cuda")
+    ws.view(torch.float32)[64:].fill_(float("nan"))
+    y = torch.full((s.S, s.fp, s.oh, s.ow), float("nan"), device="cuda")
+    dx = torch.full((s.S, s.f, s.h, s.w), float("nan"), device="cuda")
+    dw = torch.full((s.fp, s.f, s.kh, s.kw), float("nan"), device="cuda")
+    # a workspace that is too small is refused and the plan keeps its basis
+    before = fc.conv_plan_tile_basis(p)
+    with pytest.raises(fc.FftConvError):
+        fc.conv_plan_tune_tiling(p, xd, wd, dyd, y, dx, dw, ws[:1024], reps=1)
+    assert fc.conv_plan_tile_basis(p) == before
+    chosen, times = fc.conv_plan_tune_tiling(p, xd, wd, dyd, y, dx, dw, ws[:need], reps=2)
+    torch.cuda.synchronize()
+    admissible = [b for b in (8, 16, 32, 64) if b < s.n and b >= max(s.kh, s.kw)]
+    if s.n <= 128:
+        admissible = [0] + admissible
+    assert sorted(times) == sorted(admissible)
+    assert chosen in times and times[chosen] == min(times.values())
+    assert fc.conv_plan_tile_basis(p) == chosen
+    assert fc.conv_plan_status(p) == 0
+    eff = [fc.conv_plan_pass_math(p, k) for k in range(3)]
+    ref = (oracle.fprop(x, w), oracle.bprop(dy, w, s.h, s.w), oracle.accgrad(dy, x, s.kh, s.kw))
+    for k, (got, r) in enumerate(zip((y, dx, dw), ref)):           # results of the last candidate
+        assert relerr(got.cpu().numpy().astype(np.float64), r) <= TOL[eff[k]], k
+    y.fill_(float("nan"))
+    fc.conv_fprop(p, xd, wd, y)                                     # the plan is ready to use
+    torch.cuda.synchronize()
+    assert relerr(y.cpu().numpy().astype(np.float64), ref[0]) <= TOL[fc.conv_plan_pass_math(p, 0)]
+    fc.conv_plan_destroy(p)
