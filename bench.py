@@ -54,42 +54,42 @@ MAX_BLOCKS = 400
 NCU_TRAFFIC_SOURCE = {
     "profile": "profiles/dram_traffic_per_launch_three_layer_configs.md",
     "ncu": "dram__bytes_read.sum + dram__bytes_write.sum, default cache control (caches flushed before each launch)",
-    "kernel_sources_sha256": "0bfc9cf5c90ef46238574e7b62b96c70c93ba94eca4fea4b7da562cf5dbea20a",
+    "kernel_sources_sha256": "f39e8b7a1cbb20c73f6428c3ab5d1c54ecb3f5861bb54acc6297c190d03431f2",
 }
 NCU_TRAFFIC = {
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/fprop": 53.9e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/fprop": 46.5e6,
-    "mid_S128_f96_fp256_31x31_k5/bin_contraction/fprop": 226.8e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/fprop": 193.7e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/bprop": 186.7e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/bprop": 47.1e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/fprop": 54.0e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/fprop": 46.8e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/fprop": 226.1e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/fprop": 193.3e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/bprop": 187.2e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/bprop": 48.9e6,
     "mid_S128_f96_fp256_31x31_k5/bin_contraction/bprop": 261.4e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/bprop": 54.4e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_both_operands/accgrad": 287.6e6,
-    "mid_S128_f96_fp256_31x31_k5/bin_contraction/accgrad": 239.8e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/accgrad": 101.4e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/fprop": 227.5e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/fprop": 9.2e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/fprop": 280.1e6,
-    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/fprop": 188.1e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/bprop": 54.5e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_both_operands/accgrad": 287.4e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/accgrad": 241.2e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/accgrad": 101.2e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/fprop": 227.1e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/fprop": 9.1e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/fprop": 279.6e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/fprop": 188.2e6,
     "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/bprop": 182.7e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/bprop": 9.2e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/bprop": 280.2e6,
-    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/bprop": 217.6e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_both_operands/accgrad": 457.7e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/bprop": 9.1e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/bprop": 280.0e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/bprop": 217.7e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_both_operands/accgrad": 457.5e6,
     "largek_S128_f64_fp64_64x64_k11/bin_contraction/accgrad": 313.7e6,
     "largek_S128_f64_fp64_64x64_k11/c2r_ifft/accgrad": 67.2e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/fprop": 38.9e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/fprop": 113.4e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/fprop": 39.2e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/fprop": 113.5e6,
     "deep_S128_f384_fp384_13x13_k3/bin_contraction/fprop": 225.1e6,
-    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/fprop": 56.8e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/bprop": 26.0e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/bprop": 113.2e6,
-    "deep_S128_f384_fp384_13x13_k3/bin_contraction/bprop": 224.9e6,
-    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/bprop": 56.8e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_both_operands/accgrad": 115.2e6,
-    "deep_S128_f384_fp384_13x13_k3/bin_contraction/accgrad": 195.1e6,
-    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/accgrad": 172.0e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/fprop": 56.7e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/bprop": 26.1e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/bprop": 113.4e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/bprop": 225.0e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/bprop": 56.7e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_both_operands/accgrad": 114.6e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/accgrad": 195.8e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/accgrad": 171.9e6,
 }
 
 
