@@ -54,42 +54,42 @@ MAX_BLOCKS = 400
 NCU_TRAFFIC_SOURCE = {
     "profile": "profiles/dram_traffic_per_launch_three_layer_configs.md",
     "ncu": "dram__bytes_read.sum + dram__bytes_write.sum, default cache control (caches flushed before each launch)",
-    "kernel_sources_sha256": "f39e8b7a1cbb20c73f6428c3ab5d1c54ecb3f5861bb54acc6297c190d03431f2",
+    "kernel_sources_sha256": "c769041ab80b629239de641f6bdc0dada51fecdde9b076f02f80045d2411668f",
 }
 NCU_TRAFFIC = {
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/fprop": 54.0e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/fprop": 46.8e6,
-    "mid_S128_f96_fp256_31x31_k5/bin_contraction/fprop": 226.1e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/fprop": 193.3e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/bprop": 187.2e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/bprop": 48.9e6,
-    "mid_S128_f96_fp256_31x31_k5/bin_contraction/bprop": 261.4e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/bprop": 54.5e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_both_operands/accgrad": 287.4e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/fprop": 54.1e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/fprop": 46.3e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/fprop": 225.8e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/fprop": 193.8e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/bprop": 186.3e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/bprop": 47.0e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/bprop": 261.3e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/bprop": 54.6e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_both_operands/accgrad": 286.7e6,
     "mid_S128_f96_fp256_31x31_k5/bin_contraction/accgrad": 241.2e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/accgrad": 101.2e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/fprop": 227.1e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/fprop": 9.1e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/fprop": 279.6e6,
-    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/fprop": 188.2e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/bprop": 182.7e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/bprop": 9.1e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/bprop": 280.0e6,
-    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/bprop": 217.7e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_both_operands/accgrad": 457.5e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/accgrad": 313.7e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/accgrad": 101.3e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/fprop": 227.5e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/fprop": 8.9e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/fprop": 280.7e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/fprop": 189.3e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/bprop": 183.5e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/bprop": 9.2e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/bprop": 279.5e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/bprop": 217.9e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_both_operands/accgrad": 457.4e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/accgrad": 313.8e6,
     "largek_S128_f64_fp64_64x64_k11/c2r_ifft/accgrad": 67.2e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/fprop": 39.2e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/fprop": 113.5e6,
-    "deep_S128_f384_fp384_13x13_k3/bin_contraction/fprop": 225.1e6,
-    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/fprop": 56.7e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/fprop": 41.3e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/fprop": 113.7e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/fprop": 225.0e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/fprop": 56.8e6,
     "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/bprop": 26.1e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/bprop": 113.4e6,
-    "deep_S128_f384_fp384_13x13_k3/bin_contraction/bprop": 225.0e6,
-    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/bprop": 56.7e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_both_operands/accgrad": 114.6e6,
-    "deep_S128_f384_fp384_13x13_k3/bin_contraction/accgrad": 195.8e6,
-    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/accgrad": 171.9e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/bprop": 113.2e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/bprop": 225.2e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/bprop": 56.8e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_both_operands/accgrad": 114.8e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/accgrad": 195.5e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/accgrad": 172.9e6,
 }
 
 
