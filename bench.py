@@ -5,7 +5,7 @@ of one layer (all kernels of each pass) on seeded synthetic tensors.
     python bench.py [--gpus N] [--steps K] [--warmup W]      # the whole contract, one JSON line
     python bench.py --config 1 ...                           # one layer config only (0 tiny, 1 mid, 2 large-kernel, 3 deep)
     python bench.py --shape S,f,fp,h,w,kh,kw,n [--tile t]    # a layer shape of your own
-    python bench.py --sweep-only --sweep-points 1000 --sweep-budget 900 --sweep-out gpurun_out/sweep.jsonl
+    python bench.py --sweep-only --sweep-points 1000 --sweep-budget 900 --sweep-out sweep.jsonl
     python bench.py --fft2d | --fft1d                        # throughput of the bare transforms
     python bench.py --impl reference ...                     # the float64 CPU oracle on the host cores
 

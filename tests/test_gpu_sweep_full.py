@@ -1,7 +1,7 @@
 """The whole parameter sweep (workload 5) against the oracle -- an opt-in, long run.
 
     python -m pytest tests/test_gpu_sweep_full.py -m gpu -q --sweep-points 1000 \
-        --sweep-budget 1500 --sweep-out gpurun_out/sweep_parity.jsonl [--sweep-tile auto]
+        --sweep-budget 1500 --sweep-out sweep_parity.jsonl [--sweep-tile auto]
 
 Every seeded point of the sweep, all three passes, default math mode: small
 points are compared element by element, the others at seeded sampled
