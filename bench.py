@@ -54,42 +54,42 @@ MAX_BLOCKS = 400
 NCU_TRAFFIC_SOURCE = {
     "profile": "profiles/dram_traffic_per_launch_three_layer_configs.md",
     "ncu": "dram__bytes_read.sum + dram__bytes_write.sum, default cache control (caches flushed before each launch)",
-    "kernel_sources_sha256": "c769041ab80b629239de641f6bdc0dada51fecdde9b076f02f80045d2411668f",
+    "kernel_sources_sha256": "8093a5cb9b8182a7ddaf386527d8b43b04cee811388ada43c98902d481bfc6b8",
 }
 NCU_TRAFFIC = {
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/fprop": 54.1e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/fprop": 46.3e6,
-    "mid_S128_f96_fp256_31x31_k5/bin_contraction/fprop": 225.8e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/fprop": 193.8e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/bprop": 186.3e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/bprop": 47.0e6,
-    "mid_S128_f96_fp256_31x31_k5/bin_contraction/bprop": 261.3e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/bprop": 54.6e6,
-    "mid_S128_f96_fp256_31x31_k5/r2c_fft_both_operands/accgrad": 286.7e6,
-    "mid_S128_f96_fp256_31x31_k5/bin_contraction/accgrad": 241.2e6,
-    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/accgrad": 101.3e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/fprop": 227.5e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/fprop": 8.9e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/fprop": 280.7e6,
-    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/fprop": 189.3e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/bprop": 183.5e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/bprop": 9.2e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/bprop": 279.5e6,
-    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/bprop": 217.9e6,
-    "largek_S128_f64_fp64_64x64_k11/r2c_fft_both_operands/accgrad": 457.4e6,
-    "largek_S128_f64_fp64_64x64_k11/bin_contraction/accgrad": 313.8e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/fprop": 55.0e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/fprop": 40.5e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/fprop": 226.1e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/fprop": 194.6e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_first_operand/bprop": 186.8e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_small_planes/bprop": 41.0e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/bprop": 261.7e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/bprop": 54.4e6,
+    "mid_S128_f96_fp256_31x31_k5/r2c_fft_both_operands/accgrad": 286.6e6,
+    "mid_S128_f96_fp256_31x31_k5/bin_contraction/accgrad": 240.9e6,
+    "mid_S128_f96_fp256_31x31_k5/c2r_ifft/accgrad": 101.2e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/fprop": 227.2e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/fprop": 7.9e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/fprop": 280.0e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/fprop": 187.9e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_first_operand/bprop": 183.1e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_small_planes/bprop": 7.8e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/bprop": 280.5e6,
+    "largek_S128_f64_fp64_64x64_k11/c2r_ifft/bprop": 217.3e6,
+    "largek_S128_f64_fp64_64x64_k11/r2c_fft_both_operands/accgrad": 457.9e6,
+    "largek_S128_f64_fp64_64x64_k11/bin_contraction/accgrad": 313.7e6,
     "largek_S128_f64_fp64_64x64_k11/c2r_ifft/accgrad": 67.2e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/fprop": 41.3e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/fprop": 113.7e6,
-    "deep_S128_f384_fp384_13x13_k3/bin_contraction/fprop": 225.0e6,
-    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/fprop": 56.8e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/bprop": 26.1e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/bprop": 113.2e6,
-    "deep_S128_f384_fp384_13x13_k3/bin_contraction/bprop": 225.2e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/fprop": 38.4e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/fprop": 100.3e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/fprop": 224.6e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/fprop": 56.7e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_first_operand/bprop": 25.3e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_small_planes/bprop": 99.6e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/bprop": 224.9e6,
     "deep_S128_f384_fp384_13x13_k3/c2r_ifft/bprop": 56.8e6,
-    "deep_S128_f384_fp384_13x13_k3/r2c_fft_both_operands/accgrad": 114.8e6,
-    "deep_S128_f384_fp384_13x13_k3/bin_contraction/accgrad": 195.5e6,
-    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/accgrad": 172.9e6,
+    "deep_S128_f384_fp384_13x13_k3/r2c_fft_both_operands/accgrad": 114.7e6,
+    "deep_S128_f384_fp384_13x13_k3/bin_contraction/accgrad": 196.1e6,
+    "deep_S128_f384_fp384_13x13_k3/c2r_ifft/accgrad": 172.3e6,
 }
 
 

@@ -62,6 +62,7 @@ struct SmallParams {
     long long tasks;            // R * cblocks * groups
     int pitch;                  // floats per plane in shared memory (odd)
     int concurrent;             // launched to run beside its predecessor: do not wait for it (see launch_r2c_small)
+    int skip_conj;              // do not store the bins (kx > n/2, ky in {0, n/2}): the contraction leaves them out
 };
 
 template <int N, int KW>
@@ -146,6 +147,8 @@ r2c_small_kernel(const SmallParams p) {
         for (int j = 0; j < SMALL_KY; ++j) {
             if (j >= kys) break;
             float* o = o0 + (size_t)j * mat;
+            // rows ky = 0 and ky = n/2: the bins kx > n/2 are conjugates of kept bins (GemmParams::herm_n)
+            const bool herm_row = p.skip_conj && (ky0 + j == 0 || ky0 + j == N / 2);
             static_for<NQ>([&](auto KX0) {
                 constexpr int kx0 = decltype(KX0)::value;
                 float Pr[4] = {0.0f, 0.0f, 0.0f, 0.0f}, Pi[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -168,8 +171,12 @@ r2c_small_kernel(const SmallParams p) {
                     float* q = o + (size_t)kx0 * step;
                     q[0] = ar + cr;                 q[part] = ai + ci;                       // m = 0
                     q[quarter] = br + di;           q[quarter + part] = bi - dr;             // m = 1: P0 - iP1 - P2 + iP3
-                    q[2 * quarter] = ar - cr;       q[2 * quarter + part] = ai - ci;         // m = 2
-                    q[3 * quarter] = br - di;       q[3 * quarter + part] = bi + dr;         // m = 3: P0 + iP1 - P2 - iP3
+                    if (kx0 == 0 || !herm_row) {
+                        q[2 * quarter] = ar - cr;   q[2 * quarter + part] = ai - ci;         // m = 2
+                    }
+                    if (!herm_row) {
+                        q[3 * quarter] = br - di;   q[3 * quarter + part] = bi + dr;         // m = 3: P0 + iP1 - P2 - iP3
+                    }
                 }
             });
         }
@@ -221,7 +228,7 @@ static cudaError_t launch_r2c_small_n(const SmallParams& p, cudaStream_t st, boo
 // additionally start without waiting for that kernel, so that the two run side by side (the wait
 // moves to the end of this kernel, which keeps the chain of dependent launches ordered).
 static cudaError_t launch_r2c_small(int n, const FftParams& f, int ky_begin, int ky_end, cudaStream_t st,
-                                    bool overlap = false, bool concurrent = false) {
+                                    bool overlap = false, bool concurrent = false, bool skip_conj = false) {
     if (!small_supported(n, f.h, f.w) || f.win) return cudaErrorNotSupported;
     if (ky_begin < 0 || ky_end > n / 2 + 1 || ky_begin >= ky_end) return cudaErrorInvalidValue;
     SmallParams p{};
@@ -240,6 +247,7 @@ static cudaError_t launch_r2c_small(int n, const FftParams& f, int ky_begin, int
     p.tasks = blocks * p.groups;
     p.pitch = (f.h * f.w) | 1;
     p.concurrent = (overlap && concurrent) ? 1 : 0;
+    p.skip_conj = skip_conj ? 1 : 0;
     switch (n) {
         case 8:   return launch_r2c_small_n<8>(p, st, overlap);
         case 16:  return launch_r2c_small_n<16>(p, st, overlap);

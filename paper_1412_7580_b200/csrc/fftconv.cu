@@ -283,10 +283,14 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     };
     // dep: another forward transform of this pass was launched just before; the small-plane kernel
     // then runs beside it (neither touches the other's data) and completes only after it.
+    // one-pass inverse transforms (n <= 64) rebuild the conjugate bins of the rows ky = 0 and
+    // ky = n/2 themselves, so the contraction leaves them out (and the small-plane transform,
+    // whose stores are single lines, does not write them)
+    const int herm_n = (!big && plan->n <= 64) ? plan->n : 0;
     auto forward_small = [&](const fc::FftParams& f, bool dep) -> cudaError_t {
         g_launches.fetch_add(1, std::memory_order_relaxed);
         const bool conc = dep && !big && !timing;
-        return fc::launch_r2c_small(plan->n, f, 0, plan->n / 2 + 1, st, conc, conc);
+        return fc::launch_r2c_small(plan->n, f, 0, plan->n / 2 + 1, st, conc, conc, herm_n != 0);
     };
     mark(0);
     const fc::FftParams fa = operand(d.a, a_in, specA), fb = operand(d.b, b_in, specB);
@@ -302,9 +306,6 @@ int run_pass(conv_plan_s* plan, int pass, const float* a_in, const float* b_in, 
     gp.transA = d.transA; gp.transB = d.transB; gp.conjA = d.conjA; gp.conjB = d.conjB;
     gp.wait_cycles = plan->wait_cycles;
     gp.nc = plan->n / 2 + 1;
-    // one-pass inverse transforms (n <= 64) rebuild the conjugate bins of the rows ky = 0 and
-    // ky = n/2 themselves, so the contraction leaves them out
-    const int herm_n = (!big && plan->n <= 64) ? plan->n : 0;
 
     const int nc = plan->n / 2 + 1;
     const int chunks = (want_chunks && small_b) ? (plan->filter_chunks < nc ? plan->filter_chunks : nc) : 1;
